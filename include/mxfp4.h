@@ -1,0 +1,137 @@
+/*
+ * mxfp4.h - C ABI of the B200 (sm_100a) MXFP4 linear-layer backward library.
+ *
+ * The library computes the backward GEMMs of a linear layer y = x W^T,
+ *     dX = dY W      (dgrad, reduce over out-features m)
+ *     dW = dY^T X    (wgrad, reduce over tokens b)
+ * in MXFP4: each operand goes through a blockwise random Hadamard transform
+ * along the reduction dimension (one shared sign vector), is quantised to
+ * E2M1 values with one E8M0 scale per 32 contiguous elements, and the
+ * products run as block-scaled FP4 tensor-core GEMMs ("Training LLMs with
+ * MXFP4", Algorithms 1-3).
+ *
+ * Conventions for every call
+ *   - All data pointers are DEVICE pointers owned by the caller.  Nothing the
+ *     caller can see is allocated by the library; it never synchronises the
+ *     stream (except mxfp4_device_status) and enqueues all work on the CUDA
+ *     stream passed as `cuda_stream` (a cudaStream_t cast to void*, NULL = the
+ *     legacy default stream).
+ *   - Tensors are row-major.  bf16 data, codes and scales must be 16-byte
+ *     aligned; leading dimensions must keep every row 16-byte aligned.
+ *   - Return value: MXFP4_OK or an error code; on error nothing was enqueued.
+ *     Invalid arguments are reported as errors, never as undefined behaviour.
+ *   - Inputs must be finite.  A block containing Inf/NaN gets scale byte 255.
+ *   - Same inputs + same seed => bit-identical outputs.
+ */
+#ifndef MXFP4_B200_H_
+#define MXFP4_B200_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#if defined(__GNUC__)
+#define MXFP4_API __attribute__((visibility("default")))
+#else
+#define MXFP4_API
+#endif
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef enum {
+    MXFP4_OK = 0,
+    MXFP4_ERR_NULL = 1,       /* a required pointer is NULL */
+    MXFP4_ERR_SHAPE = 2,      /* a dimension is zero/negative or not divisible as required */
+    MXFP4_ERR_ALIGN = 3,      /* a pointer or leading dimension breaks the 16-byte rule */
+    MXFP4_ERR_BAD_G = 4,      /* g not in {0, 32, 64, 128, 256} or does not divide the reduce length */
+    MXFP4_ERR_MODE = 5,       /* unknown rounding / layout / dtype selector */
+    MXFP4_ERR_WORKSPACE = 6,  /* workspace NULL, misaligned or too small */
+    MXFP4_ERR_DEVICE = 7,     /* current device is not sm_100 */
+    MXFP4_ERR_CUDA = 8,       /* a CUDA runtime / driver call failed */
+    MXFP4_ERR_TIMEOUT = 9     /* a bounded device-side wait expired (see mxfp4_device_status) */
+} mxfp4_status;
+
+/* rounding: Algorithm 2 (3/4 pre-scale + stochastic rounding) or Algorithm 1 (OCP nearest rounding) */
+enum { MXFP4_ROUND_SR = 0, MXFP4_ROUND_RN = 1 };
+/* scale layout: LINEAR = [rows, K/32] row-major bytes.
+ * NATIVE = the tcgen05 scale-factor tiling consumed by mxfp4_gemm: rows padded to 128, K/32 padded to 4;
+ * byte of (row r, block k) at ((r/128)*ceil(K/128) + k/4)*512 + (r%32)*16 + ((r%128)/32)*4 + k%4. */
+enum { MXFP4_SF_LINEAR = 0, MXFP4_SF_NATIVE = 1 };
+enum { MXFP4_OUT_BF16 = 0, MXFP4_OUT_FP32 = 1 };
+
+/*
+ * Blockwise RHT + MXFP4 quantisation of one GEMM operand
+ * (Algorithm 3 lines 3-6 followed by Algorithm 2, or Algorithm 1 when rounding = RN).
+ *
+ *   x          bf16 [rows, cols], leading dimension ld elements (ld >= cols, ld % 8 == 0).
+ *   reduce_dim 1: the reduction (K) dimension is `cols` (contiguous).  Output operand is [rows, K = cols].
+ *              0: the reduction dimension is `rows`; the output is the TRANSPOSED operand [cols, K = rows]
+ *                 (the views of W, dY^T and X^T in Algorithm 3).
+ *   g          RHT block size along K: 0 = no transform, else 32/64/128/256; K % max(g, 32) == 0
+ *              (K % 128 == 0 for the NATIVE scale layout).  Every contiguous g-chunk v becomes
+ *              v diag(S) H_g / sqrt(g), H_g the Sylvester Hadamard matrix (Eq. 4), S derived from `seed`.
+ *   rounding   MXFP4_ROUND_SR: per 32 values, shared_exp = floor(log2 amax) - 2, then each value is
+ *              multiplied by 3/4, divided by 2^shared_exp and stochastically rounded to E2M1 with an 8-bit
+ *              Philox4x32-10 draw keyed on (seed, stream_tag, element index).  MXFP4_ROUND_RN: nearest
+ *              rounding (ties to even, saturating at 6) of value / 2^shared_exp, no pre-scale.
+ *   seed       drives the sign vector (shared by every operand quantised with the same seed) and SR.
+ *   stream_tag separates the SR noise of different operands that share a seed (they must differ between
+ *              the two operands of one GEMM for the product to be unbiased, Lemma 3.1).
+ *   codes      out, [R, K/2] bytes, two E2M1 codes per byte, even k in the low nibble (R = output rows).
+ *   scales     out, E8M0 bytes (value 2^(byte-127)) in `sf_layout`; mxfp4_scale_bytes() gives the size.
+ */
+MXFP4_API mxfp4_status mxfp4_rht_sr_quantize(const void* x, int64_t rows, int64_t cols, int64_t ld, int reduce_dim,
+                                   int g, int rounding, uint64_t seed, uint32_t stream_tag,
+                                   uint8_t* codes, uint8_t* scales, int sf_layout, void* cuda_stream);
+
+/*
+ * The transform alone (Algorithm 3 lines 3-6; Section 3.2): writes the fp32 values that the quantiser
+ * rounds, y [R, K] row-major, same `reduce_dim`/`g`/`seed` meaning as above.  For inspection and tests.
+ */
+MXFP4_API mxfp4_status mxfp4_rht(const void* x, int64_t rows, int64_t cols, int64_t ld, int reduce_dim,
+                       int g, uint64_t seed, float* y, void* cuda_stream);
+
+/*
+ * Block-scaled FP4 GEMM (MXFP4_GEMM of Algorithm 3 lines 7-8, with the 16/9 of lines 10-11 as alpha):
+ *     C[M, N] = alpha * sum_k deq(A)[i, k] * deq(B)[j, k],   deq = E2M1 value * 2^(scale byte - 127)
+ *   A_codes [M, K/2], B_codes [N, K/2] packed as above; A_scales / B_scales in the NATIVE layout
+ *   (sf_layout must be MXFP4_SF_NATIVE); K % 128 == 0; N % 8 == 0.
+ *   C row-major with leading dimension ldc elements, bf16 or fp32 per out_dtype; fp32 accumulation.
+ */
+MXFP4_API mxfp4_status mxfp4_gemm(const uint8_t* A_codes, const uint8_t* A_scales,
+                        const uint8_t* B_codes, const uint8_t* B_scales,
+                        int64_t M, int64_t N, int64_t K, int sf_layout, float alpha,
+                        void* C, int64_t ldc, int out_dtype, void* cuda_stream);
+
+/* Bytes of device workspace mxfp4_linear_backward needs for these shapes (codes + scales of the four
+ * quantised operands). */
+MXFP4_API size_t mxfp4_linear_backward_workspace(int64_t b, int64_t m, int64_t n);
+
+/*
+ * Algorithm 3: MXFP4 linear-layer backward with the blockwise RHT.
+ *   dY bf16 [b, m], X bf16 [b, n], W bf16 [m, n]  ->  dX [b, n], dW [m, n] (bf16 or fp32, dense).
+ *   g divides m and b (the two reduction lengths); with g = 0, m % 128 == 0 and b % 128 == 0.
+ *   The four operand views are quantised with stream tags 1..4 (dY, W^T, dY^T, X^T) and one shared sign
+ *   vector; dX = alpha Q1 Q2^T, dW = alpha Q3 Q4^T with alpha = 16/9 iff rounding = SR.
+ *   workspace: device scratch of at least mxfp4_linear_backward_workspace() bytes, 256-byte aligned;
+ *   its contents are overwritten.  Calls sharing a workspace must be stream-ordered.
+ */
+MXFP4_API mxfp4_status mxfp4_linear_backward(const void* dY, const void* X, const void* W,
+                                   int64_t b, int64_t m, int64_t n, int g, int rounding, uint64_t seed,
+                                   void* dX, void* dW, int out_dtype,
+                                   void* workspace, size_t workspace_bytes, void* cuda_stream);
+
+/* Size in bytes of a scale tensor for an operand [rows, K] in the given layout (NATIVE is padded). */
+MXFP4_API size_t mxfp4_scale_bytes(int64_t rows, int64_t K, int sf_layout);
+
+/* Synchronises `cuda_stream`, then reads and clears the device status word that kernels set when a
+ * bounded wait expires.  Returns MXFP4_OK, MXFP4_ERR_TIMEOUT or MXFP4_ERR_CUDA.  The only call that blocks. */
+MXFP4_API mxfp4_status mxfp4_device_status(void* cuda_stream);
+
+MXFP4_API const char* mxfp4_status_string(mxfp4_status status);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* MXFP4_B200_H_ */

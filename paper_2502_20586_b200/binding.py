@@ -1,0 +1,137 @@
+"""Thin Python binding of the C-ABI library (include/mxfp4.h): argument marshalling only.
+
+Every step of the method runs in the CUDA kernels behind ``libmxfp4_b200.so``; torch is used for device
+memory and streams.  There is no CPU fallback: if the library has not been built this module fails to import.
+"""
+import ctypes as C
+import os
+
+import torch
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+LIB_PATH = os.path.join(_HERE, "libmxfp4_b200.so")
+if not os.path.exists(LIB_PATH):
+    raise ImportError(f"{LIB_PATH} is missing: build it with `python -m paper_2502_20586_b200.build` "
+                      "(there is no CPU fallback)")
+_lib = C.CDLL(LIB_PATH)
+
+OK = 0
+ROUND_SR, ROUND_RN = 0, 1
+SF_LINEAR, SF_NATIVE = 0, 1
+OUT_BF16, OUT_FP32 = 0, 1
+
+_vp, _i64, _u64, _u32, _int, _sz = C.c_void_p, C.c_int64, C.c_uint64, C.c_uint32, C.c_int, C.c_size_t
+_lib.mxfp4_rht_sr_quantize.argtypes = [_vp, _i64, _i64, _i64, _int, _int, _int, _u64, _u32, _vp, _vp, _int, _vp]
+_lib.mxfp4_rht_sr_quantize.restype = _int
+_lib.mxfp4_rht.argtypes = [_vp, _i64, _i64, _i64, _int, _int, _u64, _vp, _vp]
+_lib.mxfp4_rht.restype = _int
+_lib.mxfp4_gemm.argtypes = [_vp, _vp, _vp, _vp, _i64, _i64, _i64, _int, C.c_float, _vp, _i64, _int, _vp]
+_lib.mxfp4_gemm.restype = _int
+_lib.mxfp4_linear_backward_workspace.argtypes = [_i64, _i64, _i64]
+_lib.mxfp4_linear_backward_workspace.restype = _sz
+_lib.mxfp4_linear_backward.argtypes = [_vp, _vp, _vp, _i64, _i64, _i64, _int, _int, _u64, _vp, _vp, _int, _vp, _sz, _vp]
+_lib.mxfp4_linear_backward.restype = _int
+_lib.mxfp4_scale_bytes.argtypes = [_i64, _i64, _int]
+_lib.mxfp4_scale_bytes.restype = _sz
+_lib.mxfp4_device_status.argtypes = [_vp]
+_lib.mxfp4_device_status.restype = _int
+_lib.mxfp4_status_string.argtypes = [_int]
+_lib.mxfp4_status_string.restype = C.c_char_p
+
+EXPORTS = ["mxfp4_rht_sr_quantize", "mxfp4_rht", "mxfp4_gemm", "mxfp4_linear_backward_workspace",
+           "mxfp4_linear_backward", "mxfp4_scale_bytes", "mxfp4_device_status", "mxfp4_status_string"]
+
+
+class MxFp4Error(RuntimeError):
+    def __init__(self, code: int):
+        self.code = code
+        super().__init__(f"mxfp4 error {code}: {_lib.mxfp4_status_string(code).decode()}")
+
+
+def _check(code: int):
+    if code != OK:
+        raise MxFp4Error(code)
+
+
+def _stream() -> int:
+    return torch.cuda.current_stream().cuda_stream
+
+
+def _ptr(t) -> int:
+    return 0 if t is None else t.data_ptr()
+
+
+def lib():
+    """The raw ctypes handle (tests use it to probe error codes with arbitrary arguments)."""
+    return _lib
+
+
+def mxfp4_scale_bytes(rows: int, K: int, sf_layout: int = SF_NATIVE) -> int:
+    return int(_lib.mxfp4_scale_bytes(rows, K, sf_layout))
+
+
+def mxfp4_rht_sr_quantize(x: torch.Tensor, reduce_dim: int, g: int, seed: int, stream_tag: int = 0,
+                          rounding: int = ROUND_SR, sf_layout: int = SF_NATIVE, codes=None, scales=None):
+    """x: bf16 [rows, cols] on the GPU (row stride = x.stride(0)).  Returns (codes [R, K/2] u8, scales u8 flat)."""
+    assert x.is_cuda and x.dtype == torch.bfloat16 and x.dim() == 2 and x.stride(1) == 1
+    rows, cols = x.shape
+    R, K = (rows, cols) if reduce_dim == 1 else (cols, rows)
+    if codes is None:
+        codes = torch.empty((R, K // 2), dtype=torch.uint8, device=x.device)
+    if scales is None:
+        scales = torch.empty(mxfp4_scale_bytes(R, K, sf_layout), dtype=torch.uint8, device=x.device)
+    _check(_lib.mxfp4_rht_sr_quantize(_ptr(x), rows, cols, x.stride(0), reduce_dim, g, rounding, seed, stream_tag,
+                                      _ptr(codes), _ptr(scales), sf_layout, _stream()))
+    return codes, scales
+
+
+def mxfp4_rht(x: torch.Tensor, reduce_dim: int, g: int, seed: int, y=None):
+    """The transform alone: fp32 [R, K] with K the reduction dimension."""
+    assert x.is_cuda and x.dtype == torch.bfloat16 and x.dim() == 2 and x.stride(1) == 1
+    rows, cols = x.shape
+    R, K = (rows, cols) if reduce_dim == 1 else (cols, rows)
+    if y is None:
+        y = torch.empty((R, K), dtype=torch.float32, device=x.device)
+    _check(_lib.mxfp4_rht(_ptr(x), rows, cols, x.stride(0), reduce_dim, g, seed, _ptr(y), _stream()))
+    return y
+
+
+def mxfp4_gemm(A_codes, A_scales, B_codes, B_scales, alpha: float = 1.0, out_dtype: int = OUT_BF16, C_out=None):
+    """C[M, N] = alpha * deq(A) deq(B)^T; codes [M, K/2] / [N, K/2] u8, scales in the native layout."""
+    M, K2 = A_codes.shape
+    N, K2b = B_codes.shape
+    assert K2 == K2b
+    if C_out is None:
+        C_out = torch.empty((M, N), dtype=torch.float32 if out_dtype == OUT_FP32 else torch.bfloat16, device=A_codes.device)
+    _check(_lib.mxfp4_gemm(_ptr(A_codes), _ptr(A_scales), _ptr(B_codes), _ptr(B_scales), M, N, 2 * K2, SF_NATIVE,
+                           alpha, _ptr(C_out), C_out.stride(0), out_dtype, _stream()))
+    return C_out
+
+
+def mxfp4_linear_backward_workspace(b: int, m: int, n: int) -> int:
+    return int(_lib.mxfp4_linear_backward_workspace(b, m, n))
+
+
+def mxfp4_linear_backward(dY, X, W, g: int, seed: int, rounding: int = ROUND_SR, out_dtype: int = OUT_BF16,
+                          dX=None, dW=None, workspace=None):
+    """Algorithm 3: dY [b, m], X [b, n], W [m, n] bf16 (contiguous)  ->  (dX [b, n], dW [m, n])."""
+    b, m = dY.shape
+    _, n = X.shape
+    for t in (dY, X, W):
+        assert t.is_cuda and t.dtype == torch.bfloat16 and t.is_contiguous()
+    dt = torch.float32 if out_dtype == OUT_FP32 else torch.bfloat16
+    if dX is None:
+        dX = torch.empty((b, n), dtype=dt, device=dY.device)
+    if dW is None:
+        dW = torch.empty((m, n), dtype=dt, device=dY.device)
+    need = mxfp4_linear_backward_workspace(b, m, n)
+    if workspace is None:
+        workspace = torch.empty(need, dtype=torch.uint8, device=dY.device)
+    _check(_lib.mxfp4_linear_backward(_ptr(dY), _ptr(X), _ptr(W), b, m, n, g, rounding, seed, _ptr(dX), _ptr(dW),
+                                      out_dtype, _ptr(workspace), workspace.numel(), _stream()))
+    return dX, dW
+
+
+def mxfp4_device_status() -> int:
+    """Synchronises the current stream and returns the status code (0 = OK, 9 = a device-side wait timed out)."""
+    return int(_lib.mxfp4_device_status(_stream()))

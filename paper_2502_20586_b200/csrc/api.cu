@@ -1,0 +1,232 @@
+// C-ABI entry points (include/mxfp4.h): argument validation, tensor-map set-up and kernel launches.
+#include <cuda.h>
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+#include <mutex>
+
+#include "../../include/mxfp4.h"
+#include "kernels.h"
+#include "ptx.cuh"
+
+namespace {
+
+using mx::GemmArgs;
+using mx::QuantArgs;
+
+typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*, const cuuint64_t*,
+                                  const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave, CUtensorMapSwizzle,
+                                  CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+struct Runtime {
+    std::once_flag once;
+    mxfp4_status status = MXFP4_OK;
+    EncodeTiledFn encode = nullptr;
+};
+Runtime g_rt;
+
+// One-time set-up: device check, driver entry point for tensor-map encoding, shared-memory opt-in.
+mxfp4_status runtime_init() {
+    std::call_once(g_rt.once, [] {
+        int dev = 0, major = 0;
+        if (cudaGetDevice(&dev) != cudaSuccess || cudaDeviceGetAttribute(&major, cudaDevAttrComputeCapabilityMajor, dev) != cudaSuccess) {
+            g_rt.status = MXFP4_ERR_CUDA;
+            return;
+        }
+        if (major != 10) {
+            g_rt.status = MXFP4_ERR_DEVICE;
+            return;
+        }
+        void* fn = nullptr;
+        cudaDriverEntryPointQueryResult qres;
+        if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &fn, cudaEnableDefault, &qres) != cudaSuccess || fn == nullptr ||
+            qres != cudaDriverEntryPointSuccess) {
+            g_rt.status = MXFP4_ERR_CUDA;
+            return;
+        }
+        g_rt.encode = reinterpret_cast<EncodeTiledFn>(fn);
+        if (mx::gemm_init() != cudaSuccess) g_rt.status = MXFP4_ERR_CUDA;
+    });
+    return g_rt.status;
+}
+
+bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
+bool valid_g(int g) { return g == 0 || g == 32 || g == 64 || g == 128 || g == 256; }
+int64_t round_up(int64_t v, int64_t a) { return (v + a - 1) / a * a; }
+
+size_t scale_bytes(int64_t rows, int64_t K, int layout) {
+    if (rows <= 0 || K <= 0) return 0;
+    if (layout == MXFP4_SF_NATIVE) return (size_t)(((rows + 127) / 128) * ((K + 127) / 128) * 512);
+    return (size_t)(rows * ((K + 31) / 32));
+}
+
+mxfp4_status check_quant(const void* x, int64_t rows, int64_t cols, int64_t ld, int reduce_dim, int g) {
+    if (x == nullptr) return MXFP4_ERR_NULL;
+    if (rows <= 0 || cols <= 0 || ld < cols) return MXFP4_ERR_SHAPE;
+    if (reduce_dim != 0 && reduce_dim != 1) return MXFP4_ERR_MODE;
+    if (!valid_g(g)) return MXFP4_ERR_BAD_G;
+    const int64_t K = reduce_dim == 1 ? cols : rows;
+    if (K % 32 != 0) return MXFP4_ERR_SHAPE;
+    if (g != 0 && K % g != 0) return MXFP4_ERR_BAD_G;
+    if (!aligned16(x) || ld % 8 != 0 || cols % 8 != 0) return MXFP4_ERR_ALIGN;
+    if (rows * cols / 32 > (int64_t)0x7FFFFFFF * 256) return MXFP4_ERR_SHAPE;
+    return MXFP4_OK;
+}
+
+// Tensor map over packed codes [rows, K/2] bytes: box = 128 bytes of K x box_rows rows, 128-byte swizzle.
+mxfp4_status make_codes_map(CUtensorMap* map, const uint8_t* codes, int64_t rows, int64_t K, int box_rows) {
+    const cuuint64_t dims[2] = {(cuuint64_t)(K / 2), (cuuint64_t)rows};
+    const cuuint64_t strides[1] = {(cuuint64_t)(K / 2)};
+    const cuuint32_t box[2] = {(cuuint32_t)mx::kGemmBKBytes, (cuuint32_t)box_rows};
+    const cuuint32_t elem_strides[2] = {1, 1};
+    const CUresult r = g_rt.encode(map, CU_TENSOR_MAP_DATA_TYPE_UINT8, 2, const_cast<uint8_t*>(codes), dims, strides, box, elem_strides,
+                                   CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                                   CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+    return r == CUDA_SUCCESS ? MXFP4_OK : MXFP4_ERR_CUDA;
+}
+
+mxfp4_status gemm_impl(const uint8_t* A_codes, const uint8_t* A_scales, const uint8_t* B_codes, const uint8_t* B_scales, int64_t M,
+                       int64_t N, int64_t K, float alpha, void* C, int64_t ldc, int out_dtype, cudaStream_t stream) {
+    GemmArgs a;
+    mxfp4_status st = make_codes_map(&a.tmap_a, A_codes, M, K, mx::kGemmBM);
+    if (st != MXFP4_OK) return st;
+    st = make_codes_map(&a.tmap_b, B_codes, N, K, mx::kGemmBN);
+    if (st != MXFP4_OK) return st;
+    a.sfa = A_scales; a.sfb = B_scales;
+    a.M = M; a.N = N; a.K = K;
+    a.alpha = alpha; a.C = C; a.ldc = ldc; a.out_fp32 = out_dtype == MXFP4_OUT_FP32;
+    return mx::launch_gemm(a, stream) == cudaSuccess ? MXFP4_OK : MXFP4_ERR_CUDA;
+}
+
+struct Workspace {
+    size_t codes[4], scales[4], total;
+};
+// Operand views of Algorithm 3: Q1 = dY [b, K=m], Q2 = W^T [n, K=m], Q3 = dY^T [m, K=b], Q4 = X^T [n, K=b].
+Workspace plan_workspace(int64_t b, int64_t m, int64_t n) {
+    const int64_t R[4] = {b, n, m, n}, K[4] = {m, m, b, b};
+    Workspace w;
+    size_t off = 0;
+    for (int i = 0; i < 4; ++i) {
+        w.codes[i] = off;
+        off += (size_t)round_up(R[i] * K[i] / 2, 1024);
+        w.scales[i] = off;
+        off += (size_t)round_up((int64_t)scale_bytes(R[i], K[i], MXFP4_SF_NATIVE), 1024);
+    }
+    w.total = off;
+    return w;
+}
+
+}  // namespace
+
+extern "C" {
+
+const char* mxfp4_status_string(mxfp4_status s) {
+    switch (s) {
+        case MXFP4_OK: return "ok";
+        case MXFP4_ERR_NULL: return "null pointer";
+        case MXFP4_ERR_SHAPE: return "bad shape";
+        case MXFP4_ERR_ALIGN: return "bad alignment";
+        case MXFP4_ERR_BAD_G: return "bad RHT block size g";
+        case MXFP4_ERR_MODE: return "bad mode selector";
+        case MXFP4_ERR_WORKSPACE: return "bad workspace";
+        case MXFP4_ERR_DEVICE: return "device is not sm_100";
+        case MXFP4_ERR_CUDA: return "CUDA call failed";
+        case MXFP4_ERR_TIMEOUT: return "device-side wait timed out";
+    }
+    return "unknown status";
+}
+
+size_t mxfp4_scale_bytes(int64_t rows, int64_t K, int sf_layout) { return scale_bytes(rows, K, sf_layout); }
+
+mxfp4_status mxfp4_rht_sr_quantize(const void* x, int64_t rows, int64_t cols, int64_t ld, int reduce_dim, int g, int rounding,
+                                   uint64_t seed, uint32_t stream_tag, uint8_t* codes, uint8_t* scales, int sf_layout,
+                                   void* cuda_stream) {
+    if (codes == nullptr || scales == nullptr) return MXFP4_ERR_NULL;
+    mxfp4_status st = check_quant(x, rows, cols, ld, reduce_dim, g);
+    if (st != MXFP4_OK) return st;
+    if (rounding != MXFP4_ROUND_SR && rounding != MXFP4_ROUND_RN) return MXFP4_ERR_MODE;
+    if (sf_layout != MXFP4_SF_LINEAR && sf_layout != MXFP4_SF_NATIVE) return MXFP4_ERR_MODE;
+    if (!aligned16(codes)) return MXFP4_ERR_ALIGN;
+    if ((st = runtime_init()) != MXFP4_OK) return st;
+    QuantArgs a{x, rows, cols, ld, reduce_dim, g, rounding, seed, stream_tag, codes, scales, sf_layout == MXFP4_SF_NATIVE, nullptr};
+    return mx::launch_quantize(a, static_cast<cudaStream_t>(cuda_stream)) == cudaSuccess ? MXFP4_OK : MXFP4_ERR_CUDA;
+}
+
+mxfp4_status mxfp4_rht(const void* x, int64_t rows, int64_t cols, int64_t ld, int reduce_dim, int g, uint64_t seed, float* y,
+                       void* cuda_stream) {
+    if (y == nullptr) return MXFP4_ERR_NULL;
+    mxfp4_status st = check_quant(x, rows, cols, ld, reduce_dim, g);
+    if (st != MXFP4_OK) return st;
+    if (!aligned16(y)) return MXFP4_ERR_ALIGN;
+    if ((st = runtime_init()) != MXFP4_OK) return st;
+    QuantArgs a{x, rows, cols, ld, reduce_dim, g, 0, seed, 0u, nullptr, nullptr, 0, y};
+    return mx::launch_rht_dump(a, static_cast<cudaStream_t>(cuda_stream)) == cudaSuccess ? MXFP4_OK : MXFP4_ERR_CUDA;
+}
+
+mxfp4_status mxfp4_gemm(const uint8_t* A_codes, const uint8_t* A_scales, const uint8_t* B_codes, const uint8_t* B_scales, int64_t M,
+                        int64_t N, int64_t K, int sf_layout, float alpha, void* C, int64_t ldc, int out_dtype, void* cuda_stream) {
+    if (!A_codes || !A_scales || !B_codes || !B_scales || !C) return MXFP4_ERR_NULL;
+    if (M <= 0 || N <= 0 || K <= 0 || K % 128 != 0 || N % 8 != 0 || ldc < N) return MXFP4_ERR_SHAPE;
+    if (M > 0x7FFFFFFF || N > 0x7FFFFFFF || K > 0x7FFFFFFF) return MXFP4_ERR_SHAPE;
+    if (sf_layout != MXFP4_SF_NATIVE) return MXFP4_ERR_MODE;
+    if (out_dtype != MXFP4_OUT_BF16 && out_dtype != MXFP4_OUT_FP32) return MXFP4_ERR_MODE;
+    if (!aligned16(A_codes) || !aligned16(B_codes) || !aligned16(A_scales) || !aligned16(B_scales) || !aligned16(C)) return MXFP4_ERR_ALIGN;
+    if (ldc % (out_dtype == MXFP4_OUT_FP32 ? 4 : 8) != 0) return MXFP4_ERR_ALIGN;
+    const mxfp4_status st = runtime_init();
+    if (st != MXFP4_OK) return st;
+    return gemm_impl(A_codes, A_scales, B_codes, B_scales, M, N, K, alpha, C, ldc, out_dtype, static_cast<cudaStream_t>(cuda_stream));
+}
+
+size_t mxfp4_linear_backward_workspace(int64_t b, int64_t m, int64_t n) {
+    if (b <= 0 || m <= 0 || n <= 0) return 0;
+    return plan_workspace(b, m, n).total;
+}
+
+mxfp4_status mxfp4_linear_backward(const void* dY, const void* X, const void* W, int64_t b, int64_t m, int64_t n, int g, int rounding,
+                                   uint64_t seed, void* dX, void* dW, int out_dtype, void* workspace, size_t workspace_bytes,
+                                   void* cuda_stream) {
+    if (!dY || !X || !W || !dX || !dW) return MXFP4_ERR_NULL;
+    if (b <= 0 || m <= 0 || n <= 0) return MXFP4_ERR_SHAPE;
+    if (!valid_g(g)) return MXFP4_ERR_BAD_G;
+    if (m % 128 != 0 || b % 128 != 0 || n % 8 != 0) return MXFP4_ERR_SHAPE;       // both reduce lengths feed the GEMM (K % 128)
+    if (g != 0 && (m % g != 0 || b % g != 0)) return MXFP4_ERR_BAD_G;
+    if (rounding != MXFP4_ROUND_SR && rounding != MXFP4_ROUND_RN) return MXFP4_ERR_MODE;
+    if (out_dtype != MXFP4_OUT_BF16 && out_dtype != MXFP4_OUT_FP32) return MXFP4_ERR_MODE;
+    if (!aligned16(dY) || !aligned16(X) || !aligned16(W) || !aligned16(dX) || !aligned16(dW)) return MXFP4_ERR_ALIGN;
+    const Workspace ws = plan_workspace(b, m, n);
+    if (workspace == nullptr || workspace_bytes < ws.total || (reinterpret_cast<uintptr_t>(workspace) & 255u) != 0) return MXFP4_ERR_WORKSPACE;
+    mxfp4_status st = runtime_init();
+    if (st != MXFP4_OK) return st;
+    cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
+    uint8_t* base = static_cast<uint8_t*>(workspace);
+    uint8_t *c[4], *s[4];
+    for (int i = 0; i < 4; ++i) { c[i] = base + ws.codes[i]; s[i] = base + ws.scales[i]; }
+    // Algorithm 3 lines 3-6: stream tags 1..4, one sign vector (same seed) for all four views.
+    const QuantArgs q[4] = {
+        {dY, b, m, m, 1, g, rounding, seed, 1u, c[0], s[0], 1, nullptr},   // dY   [b, K = m]
+        {W, m, n, n, 0, g, rounding, seed, 2u, c[1], s[1], 1, nullptr},    // W^T  [n, K = m]
+        {dY, b, m, m, 0, g, rounding, seed, 3u, c[2], s[2], 1, nullptr},   // dY^T [m, K = b]
+        {X, b, n, n, 0, g, rounding, seed, 4u, c[3], s[3], 1, nullptr},    // X^T  [n, K = b]
+    };
+    for (int i = 0; i < 4; ++i)
+        if (mx::launch_quantize(q[i], stream) != cudaSuccess) return MXFP4_ERR_CUDA;
+    // lines 7-11: two MXFP4 GEMMs; the 16/9 un-does the two 3/4 pre-scales of Algorithm 2.
+    const float alpha = rounding == MXFP4_ROUND_SR ? 16.0f / 9.0f : 1.0f;
+    st = gemm_impl(c[0], s[0], c[1], s[1], b, n, m, alpha, dX, n, out_dtype, stream);
+    if (st != MXFP4_OK) return st;
+    return gemm_impl(c[2], s[2], c[3], s[3], m, n, b, alpha, dW, n, out_dtype, stream);
+}
+
+mxfp4_status mxfp4_device_status(void* cuda_stream) {
+    if (cudaStreamSynchronize(static_cast<cudaStream_t>(cuda_stream)) != cudaSuccess) return MXFP4_ERR_CUDA;
+    unsigned int word = 0;
+    if (cudaMemcpyFromSymbol(&word, mx::g_device_status, sizeof word) != cudaSuccess) return MXFP4_ERR_CUDA;
+    if (word != 0) {
+        const unsigned int zero = 0;
+        if (cudaMemcpyToSymbol(mx::g_device_status, &zero, sizeof zero) != cudaSuccess) return MXFP4_ERR_CUDA;
+        return MXFP4_ERR_TIMEOUT;
+    }
+    return MXFP4_OK;
+}
+
+}  // extern "C"

@@ -1,0 +1,45 @@
+// Internal launch interfaces between the C-ABI layer (api.cu) and the kernel files.
+#pragma once
+#include <cuda.h>
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+namespace mx {
+
+struct QuantArgs {
+    const void* x;        // bf16 [rows, cols], leading dimension ld
+    int64_t rows, cols, ld;
+    int reduce_dim;       // 1: reduce along cols; 0: reduce along rows (transposed output)
+    int g;                // 0, 32, 64, 128, 256
+    int rounding;         // 0 SR, 1 RN
+    uint64_t seed;
+    uint32_t stream_tag;
+    uint8_t* codes;
+    uint8_t* scales;
+    int sf_native;
+    float* y_out;         // only for the transform dump
+};
+
+cudaError_t launch_quantize(const QuantArgs& a, cudaStream_t stream);
+cudaError_t launch_rht_dump(const QuantArgs& a, cudaStream_t stream);
+
+struct GemmArgs {
+    CUtensorMap tmap_a;   // codes [M, K/2] bytes, box 128 B x 128 rows, 128-byte swizzle
+    CUtensorMap tmap_b;   // codes [N, K/2] bytes, box 128 B x BN rows
+    const uint8_t* sfa;   // native scale layout
+    const uint8_t* sfb;
+    int64_t M, N, K;
+    float alpha;
+    void* C;
+    int64_t ldc;
+    int out_fp32;
+};
+
+constexpr int kGemmBM = 128;
+constexpr int kGemmBN = 256;
+constexpr int kGemmBKBytes = 128;   // 256 E2M1 elements per pipeline stage
+
+cudaError_t launch_gemm(const GemmArgs& a, cudaStream_t stream);
+cudaError_t gemm_init();            // one-time: opt in to large dynamic shared memory
+
+}  // namespace mx

@@ -1,0 +1,92 @@
+"""Host-side checks that need no GPU: the C-ABI library loads, exports every symbol the header declares,
+and rejects bad arguments with error codes before touching the device."""
+import ctypes as C
+import os
+import re
+
+import pytest
+
+ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+
+
+@pytest.fixture(scope="module")
+def lib():
+    from paper_2502_20586_b200 import build
+    build.build()
+    from paper_2502_20586_b200 import binding
+    return binding
+
+
+def test_every_declared_symbol_is_exported(lib):
+    header = open(os.path.join(ROOT, "include", "mxfp4.h")).read()
+    declared = re.findall(r"MXFP4_API\s+[\w\s\*]+?\b(mxfp4_\w+)\s*\(", header)
+    assert len(declared) >= 8
+    raw = C.CDLL(lib.LIB_PATH)
+    for name in declared:
+        assert hasattr(raw, name), name
+    assert sorted(declared) == sorted(lib.EXPORTS)
+
+
+def test_status_strings(lib):
+    raw = lib.lib()
+    seen = {raw.mxfp4_status_string(i) for i in range(10)}
+    assert len(seen) == 10 and b"ok" in seen
+
+
+def test_scale_bytes_and_workspace(lib):
+    assert lib.mxfp4_scale_bytes(256, 512, lib.SF_LINEAR) == 256 * 16
+    assert lib.mxfp4_scale_bytes(256, 512, lib.SF_NATIVE) == 2 * 4 * 512
+    assert lib.mxfp4_scale_bytes(129, 160, lib.SF_NATIVE) == 2 * 2 * 512          # padded to 128 rows x 4 blocks
+    assert lib.mxfp4_scale_bytes(0, 512, lib.SF_NATIVE) == 0
+    b, m, n = 256, 512, 512
+    need = lib.mxfp4_linear_backward_workspace(b, m, n)
+    codes = (b * m + n * m + m * b + n * b) // 2
+    assert need >= codes + codes // 16 and need % 256 == 0
+    assert lib.mxfp4_linear_backward_workspace(0, m, n) == 0
+
+
+def test_argument_validation_needs_no_device(lib):
+    raw = lib.lib()
+    P = 0x1000                                    # a fake, 16-byte aligned, never dereferenced pointer
+    q = raw.mxfp4_rht_sr_quantize
+    assert q(0, 32, 64, 64, 1, 64, 0, 0, 0, P, P, 1, 0) == 1                      # NULL
+    assert q(P, 32, 64, 64, 1, 64, 0, 0, 0, 0, P, 1, 0) == 1
+    assert q(P, 0, 64, 64, 1, 64, 0, 0, 0, P, P, 1, 0) == 2                       # shape
+    assert q(P, 32, 64, 32, 1, 64, 0, 0, 0, P, P, 1, 0) == 2                      # ld < cols
+    assert q(P, 32, 48, 48, 1, 0, 0, 0, 0, P, P, 1, 0) == 2                       # K % 32
+    assert q(P, 32, 64, 64, 1, 48, 0, 0, 0, P, P, 1, 0) == 4                      # g not a power of two
+    assert q(P, 32, 64, 64, 1, 128, 0, 0, 0, P, P, 1, 0) == 4                     # g does not divide K
+    assert q(P, 64, 64, 64, 0, 128, 0, 0, 0, P, P, 1, 0) == 4
+    assert q(P, 32, 64, 64, 2, 64, 0, 0, 0, P, P, 1, 0) == 5                      # reduce_dim
+    assert q(P, 32, 64, 64, 1, 64, 7, 0, 0, P, P, 1, 0) == 5                      # rounding
+    assert q(P, 32, 64, 64, 1, 64, 0, 0, 0, P, P, 3, 0) == 5                      # layout
+    assert q(P + 2, 32, 64, 64, 1, 64, 0, 0, 0, P, P, 1, 0) == 3                  # alignment
+    assert q(P, 32, 64, 68, 1, 64, 0, 0, 0, P, P, 1, 0) == 3                      # ld % 8
+    g = raw.mxfp4_gemm
+    assert g(0, P, P, P, 128, 128, 128, 1, 1.0, P, 128, 0, 0) == 1
+    assert g(P, P, P, P, 128, 128, 96, 1, 1.0, P, 128, 0, 0) == 2                 # K % 128
+    assert g(P, P, P, P, 128, 100, 128, 1, 1.0, P, 128, 0, 0) == 2                # N % 8
+    assert g(P, P, P, P, 128, 128, 128, 1, 1.0, P, 64, 0, 0) == 2                 # ldc < N
+    assert g(P, P, P, P, 128, 128, 128, 0, 1.0, P, 128, 0, 0) == 5                # linear scales not accepted
+    assert g(P, P, P, P, 128, 128, 128, 1, 1.0, P, 128, 9, 0) == 5
+    assert g(P, P, P + 4, P, 128, 128, 128, 1, 1.0, P, 128, 0, 0) == 3
+    lb = raw.mxfp4_linear_backward
+    assert lb(P, P, 0, 256, 512, 512, 64, 0, 0, P, P, 0, P, 1 << 30, 0) == 1
+    assert lb(P, P, P, 256, 500, 512, 64, 0, 0, P, P, 0, P, 1 << 30, 0) == 2
+    assert lb(P, P, P, 256, 512, 512, 96, 0, 0, P, P, 0, P, 1 << 30, 0) == 4
+    assert lb(P, P, P, 128, 512, 512, 256, 0, 0, P, P, 0, P, 1 << 30, 0) == 4     # g does not divide b
+    assert lb(P, P, P, 256, 512, 512, 64, 0, 0, P, P, 0, 0, 1 << 30, 0) == 6      # workspace NULL
+    assert lb(P, P, P, 256, 512, 512, 64, 0, 0, P, P, 0, P, 1024, 0) == 6         # too small
+    assert lb(P, P, P, 256, 512, 512, 64, 0, 0, P, P, 0, P + 16, 1 << 30, 0) == 6  # misaligned
+
+
+def test_binding_fails_loudly_without_library(tmp_path, monkeypatch):
+    """The product path has no CPU fallback: a missing shared library is an ImportError."""
+    import importlib.util
+    src = os.path.join(ROOT, "paper_2502_20586_b200", "binding.py")
+    dst = tmp_path / "binding_copy.py"
+    dst.write_text(open(src).read())
+    spec = importlib.util.spec_from_file_location("binding_copy", dst)
+    mod = importlib.util.module_from_spec(spec)
+    with pytest.raises(ImportError):
+        spec.loader.exec_module(mod)
