@@ -1,0 +1,360 @@
+#!/usr/bin/env python
+"""Benchmark of the MXFP4 linear-layer backward path (Algorithm 3) on B200.
+
+One "step" = dgrad + wgrad of the four linear layers of one GPT block (QKV, attention output, FC1, FC2) at the
+6.7B shapes (hidden 4096, FFN 16384, 8 x 2048 tokens, g = 128): four RHT + SR quantisations and two
+block-scaled FP4 GEMMs per layer.  Metric: backward GEMM TFLOP/s (4 b m n per layer) INCLUDING quantisation.
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--impl reference] [--config gpt_6p7b]
+
+Prints one JSON line (rank 0).  Legs of the GPU arm, all in this run:
+  value      K steps of mxfp4_linear_backward per layer, inputs resident in HBM, CUDA events, max over ranks;
+  roofline   the same step issued as its six C-ABI calls per layer with CUDA events around every call, so
+             each kernel's launch duration is measured in place; the dominant kernel (the FP4 GEMM) is
+             reported against the tensor peak, the quantisers against the HBM peak;
+  e2e        the same metric through mxfp4_linear_backward with HOST buffers: pinned host -> device copies
+             of dY, X, W and device -> host copies of dX, dW inside the timed region;
+  cpu_baseline  the CPU oracle (test infrastructure, never tuned) timed on a bounded sample (rank 0, N = 1).
+With N > 1 (torchrun) every rank runs the same workload on its own tokens (data parallel, no collective on
+this path): weak scaling, value = all ranks' FLOPs / max time.
+"""
+import argparse
+import json
+import os
+import subprocess
+import sys
+import threading
+import time
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+METRIC = "MXFP4 backward GEMM TFLOP/s incl. RHT+SR quantize"
+UNIT = "TFLOP/s"
+NOMINAL_FP4_TFLOPS = 9000.0          # dense, NVIDIA's figure; context only
+BF16_TO_FP4 = 4.0                    # nominal dense ratio 9 / 2.25 PFLOP/s
+QUANT_BYTES_PER_ELEM = 2.0 + 0.5 + 1.0 / 32.0   # bf16 in, E2M1 code + E8M0 scale out
+
+
+def load_peaks():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(path):
+        with open(path) as fh:
+            p = json.load(fh)
+        return {"hbm_gbs": p["hbm_gbs"], "bf16_burst": p["bf16_tflops"], "bf16_sustained": p["bf16_tflops_sustained"],
+                "source": "measured"}
+    return {"hbm_gbs": 6650.0, "bf16_burst": 1590.0, "bf16_sustained": 1400.0, "source": "fallback"}
+
+
+# ------------------------------------------------------------------------------------------ clock sampler
+class ClockSampler:
+    """Samples nvidia-smi clocks and throttle reasons for one GPU while a timed region runs."""
+    FIELDS = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.hw_slowdown,"
+              "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
+              "clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, index: int):
+        self.index = index
+        self.rows = []
+        self.proc = None
+        self.thread = None
+
+    def start(self):
+        try:
+            self.proc = subprocess.Popen(
+                ["nvidia-smi", f"--id={self.index}", f"--query-gpu={self.FIELDS}", "--format=csv,noheader,nounits", "-lms", "20"],
+                stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
+        except OSError:
+            self.proc = None
+            return
+        self.thread = threading.Thread(target=self._read, daemon=True)
+        self.thread.start()
+
+    def _read(self):
+        for line in self.proc.stdout:
+            self.rows.append([t.strip() for t in line.split(",")])
+
+    def stop(self):
+        if self.proc is None:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvidia-smi unavailable"]}
+        self.proc.terminate()
+        try:
+            self.proc.wait(timeout=5)
+        except subprocess.TimeoutExpired:
+            self.proc.kill()
+        sm, smax, power, reasons = [], None, [], set()
+        for r in self.rows:
+            if len(r) < 7:
+                continue
+            try:
+                sm.append(float(r[0])); smax = float(r[1]); power.append(float(r[2]))
+            except ValueError:
+                continue
+            for name, val in zip(("hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"), r[3:7]):
+                if val.lower().startswith("active"):
+                    reasons.add(name)
+        sm.sort()
+        # median over samples under load (at least half of the maximum power seen)
+        busy = sorted(s for s, p in zip([float(r[0]) for r in self.rows if len(r) >= 7], power) if p >= 0.5 * max(power)) if power else []
+        med = busy[len(busy) // 2] if busy else (sm[len(sm) // 2] if sm else None)
+        return {"sm_mhz": med, "sm_max_mhz": smax, "power_w_max": max(power) if power else None,
+                "samples": len(sm), "reasons": sorted(reasons)}
+
+
+# ------------------------------------------------------------------------------------------ reference arm
+def oracle_sample(config: str, seed: int = 0):
+    """A bounded sample of the workload for the CPU oracle: Algorithm 3 on a 4096-token slab of the
+    attention-output layer, dX in full and dW on up to 4096 sampled rows.  Returns (fn, flops, description)."""
+    import numpy as np
+    from oracle import ref
+    from paper_2502_20586_b200 import workloads as wl
+    layers, g = wl.CONFIGS[config]
+    layer = [l for l in layers if l.name in ("attn_out", "single")][0]
+    b_s = min(4096, layer.b)
+    rng = np.random.default_rng(seed)
+    std = 1e-3 if config == "single_256x512" else 1e-4
+    dY = wl.grad_like(rng, (b_s, layer.m), std)
+    X = wl.activation_like(rng, (b_s, layer.n), n_outlier_channels=8)
+    W = wl.weight_like(rng, (layer.m, layer.n))
+    dw_rows = np.sort(rng.choice(layer.m, size=min(4096, layer.m), replace=False))
+    flops = 2 * b_s * layer.n * layer.m + 2 * len(dw_rows) * layer.n * b_s
+
+    def run():
+        ref.linear_backward(dY, X, W, g, ref.ROUND_SR, seed, dw_rows=dw_rows)
+
+    desc = (f"Algorithm 3 (g={g}, SR) on a {b_s}-token slab of the {config} {layer.name} layer (n={layer.n}, m={layer.m}): "
+            f"all four operand quantisations, dX in full, dW on {len(dw_rows)} sampled rows; FLOPs = GEMM MACs x 2 actually computed")
+    return run, flops, desc, ref.num_threads()
+
+
+def run_reference(args):
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    run, flops, desc, cores = oracle_sample(args.config)
+    for _ in range(min(args.warmup, 1)):
+        run()
+    t0 = time.perf_counter()
+    for _ in range(args.steps):
+        run()
+    dt = (time.perf_counter() - t0) / args.steps
+    val = flops / dt / 1e12
+    print(json.dumps({
+        "impl": "reference", "metric": METRIC, "value": val, "unit": UNIT, "n_gpus": args.gpus, "steps": args.steps,
+        "warmup": min(args.warmup, 1), "ms_per_step": dt * 1e3, "higher_is_better": True, "scaling": "weak",
+        "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+        "config": {"workload": args.config, "sample": desc},
+        "cpu_baseline": {"value": val, "unit": UNIT, "cores": cores, "kind": "oracle", "sample": desc},
+        "e2e": {"value": val, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+    }))
+
+
+# ------------------------------------------------------------------------------------------------ GPU arm
+def run_gpu(args):
+    import torch
+    import torch.distributed as dist
+    from paper_2502_20586_b200 import binding as mx
+    from paper_2502_20586_b200 import workloads as wl
+
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    rank = int(os.environ.get("RANK", "0"))
+    local_rank = int(os.environ.get("LOCAL_RANK", "0"))
+    torch.cuda.set_device(local_rank)
+    dev = torch.device("cuda", local_rank)
+    if world > 1:
+        dist.init_process_group("nccl", device_id=dev)
+
+    def barrier():
+        if world > 1:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    peaks = load_peaks()
+    layers, g = wl.CONFIGS[args.config]
+    seed = 0
+    out_dtype = mx.OUT_BF16
+    data = []
+    for layer in layers:
+        dY, X, W = wl.layer_inputs_device(args.config, layer, seed=seed + rank, device=dev)
+        dX = torch.empty((layer.b, layer.n), dtype=torch.bfloat16, device=dev)
+        dW = torch.empty((layer.m, layer.n), dtype=torch.bfloat16, device=dev)
+        data.append((layer, dY, X, W, dX, dW))
+    ws_bytes = max(mx.mxfp4_linear_backward_workspace(l.b, l.m, l.n) for l in layers)
+    ws = torch.empty(ws_bytes, dtype=torch.uint8, device=dev)
+    flops_step = sum(l.flops for l in layers)
+    stream = torch.cuda.current_stream()
+
+    def step():
+        for (layer, dY, X, W, dX, dW) in data:
+            mx.mxfp4_linear_backward(dY, X, W, g, seed, mx.ROUND_SR, out_dtype, dX=dX, dW=dW, workspace=ws)
+
+    # ---- value: K steps, device-resident inputs
+    sampler = ClockSampler(local_rank)
+    sampler.start()
+    for _ in range(args.warmup):
+        step()
+    barrier()
+    ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    ev0.record(stream)
+    for _ in range(args.steps):
+        step()
+    ev1.record(stream)
+    barrier()
+    ms = ev0.elapsed_time(ev1) / args.steps
+    if mx.mxfp4_device_status() != 0:
+        raise RuntimeError("a device-side wait timed out during the timed region")
+
+    legs = set(args.legs.split(","))
+    kernels, calls_ms, gemm_tflops, clocks = {}, None, None, None
+    fp4_peak = BF16_TO_FP4 * peaks["bf16_sustained"]
+    if "roofline" in legs:
+        # ---- roofline: the same step as its six C-ABI calls per layer, CUDA events around each
+        # operand views of Algorithm 3: (tensor index in (dY, X, W), reduce_dim, stream tag)
+        views = ((0, 1, 1), (2, 0, 2), (0, 0, 3), (1, 0, 4))
+        bufs = []
+        for (layer, dY, X, W, dX, dW) in data:
+            ops = []
+            for (ti, rd, tag) in views:
+                t = (dY, X, W)[ti]
+                R, K = (t.shape[0], t.shape[1]) if rd == 1 else (t.shape[1], t.shape[0])
+                ops.append((t, rd, tag, torch.empty((R, K // 2), dtype=torch.uint8, device=dev),
+                            torch.empty(mx.mxfp4_scale_bytes(R, K), dtype=torch.uint8, device=dev)))
+            bufs.append(ops)
+        records = []   # (kind, layer name, start event, end event, work)
+
+        def timed(kind, name, work, fn):
+            a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            a.record(stream); fn(); b.record(stream)
+            records.append((kind, name, a, b, work))
+
+        def step_calls(record):
+            for (layer, dY, X, W, dX, dW), ops in zip(data, bufs):
+                for (t, rd, tag, codes, scales) in ops:
+                    fn = lambda t=t, rd=rd, tag=tag, codes=codes, scales=scales: mx.mxfp4_rht_sr_quantize(
+                        t, rd, g, seed, tag, mx.ROUND_SR, mx.SF_NATIVE, codes=codes, scales=scales)
+                    if record:
+                        timed("quant_row" if rd == 1 else "quant_tr", layer.name, t.numel() * QUANT_BYTES_PER_ELEM, fn)
+                    else:
+                        fn()
+                for (a, bb, out, fl) in ((0, 1, dX, 2 * layer.b * layer.n * layer.m), (2, 3, dW, 2 * layer.m * layer.n * layer.b)):
+                    fn = lambda a=a, bb=bb, out=out, ops=ops: mx.mxfp4_gemm(ops[a][3], ops[a][4], ops[bb][3], ops[bb][4],
+                                                                             16.0 / 9.0, out_dtype, C_out=out)
+                    if record:
+                        timed("gemm", layer.name, fl, fn)
+                    else:
+                        fn()
+
+        step_calls(False)
+        torch.cuda.synchronize()
+        k_roof = max(1, min(args.steps, 5))
+        for _ in range(k_roof):
+            step_calls(True)
+        barrier()
+        agg = {}
+        for kind, name, a, b, work in records:
+            d = agg.setdefault(kind, [0.0, 0.0, 0])
+            d[0] += a.elapsed_time(b) * 1e-3; d[1] += work; d[2] += 1
+        gemm_t, gemm_fl, gemm_n = agg["gemm"]
+        gemm_tflops = gemm_fl / gemm_t / 1e12
+        kernels = {}
+        for kind in ("quant_row", "quant_tr"):
+            t_, by, n_ = agg[kind]
+            kernels[kind] = {"launches": n_, "avg_ms": t_ / n_ * 1e3, "GB/s": by / t_ / 1e9,
+                             "frac_of_hbm_peak": by / t_ / 1e9 / peaks["hbm_gbs"]}
+        kernels["gemm"] = {"launches": gemm_n, "avg_ms": gemm_t / gemm_n * 1e3, "TFLOP/s": gemm_tflops,
+                           "frac_of_4x_bf16_sustained": gemm_tflops / fp4_peak,
+                           "frac_of_4x_bf16_burst": gemm_tflops / (BF16_TO_FP4 * peaks["bf16_burst"]),
+                           "frac_of_nominal_9pf": gemm_tflops / NOMINAL_FP4_TFLOPS}
+        calls_ms = sum(v[0] for v in agg.values()) / k_roof * 1e3
+
+    clocks = sampler.stop()
+    ms_e2e, h2d, d2h = None, 0, 0
+    if "e2e" in legs:
+        # ---- e2e: host buffers, copies inside the timed region
+        host = []
+        h2d = d2h = 0
+        for (layer, dY, X, W, dX, dW) in data:
+            hin = [t.cpu().pin_memory() for t in (dY, X, W)]
+            hout = [torch.empty(t.shape, dtype=t.dtype).pin_memory() for t in (dX, dW)]
+            host.append((hin, hout))
+            h2d += sum(t.numel() * t.element_size() for t in hin)
+            d2h += sum(t.numel() * t.element_size() for t in hout)
+
+        def step_e2e():
+            for (layer, dY, X, W, dX, dW), (hin, hout) in zip(data, host):
+                for dst, src in zip((dY, X, W), hin):
+                    dst.copy_(src, non_blocking=True)
+                mx.mxfp4_linear_backward(dY, X, W, g, seed, mx.ROUND_SR, out_dtype, dX=dX, dW=dW, workspace=ws)
+                for dst, src in zip(hout, (dX, dW)):
+                    dst.copy_(src, non_blocking=True)
+
+        step_e2e()
+        barrier()
+        k_e2e = max(1, min(args.steps, 5))
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record(stream)
+        for _ in range(k_e2e):
+            step_e2e()
+        e1.record(stream)
+        barrier()
+        ms_e2e = e0.elapsed_time(e1) / k_e2e
+
+    # ---- max over ranks
+    if world > 1:
+        t = torch.tensor([ms, ms_e2e or 0.0], device=dev, dtype=torch.float64)
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        ms, ms_e2e = float(t[0]), (float(t[1]) if ms_e2e else None)
+    value = world * flops_step / (ms * 1e-3) / 1e12
+    e2e_value = world * flops_step / (ms_e2e * 1e-3) / 1e12 if ms_e2e else None
+
+    cpu_baseline = None
+    if rank == 0 and world == 1 and not args.no_cpu_baseline and "e2e" in legs:
+        run, fl, desc, cores = oracle_sample(args.config)
+        t0 = time.perf_counter()
+        run()
+        dt = time.perf_counter() - t0
+        cpu_baseline = {"value": fl / dt / 1e12, "unit": UNIT, "cores": cores, "kind": "oracle", "sample": desc, "seconds": dt}
+
+    if rank == 0:
+        print(json.dumps({
+            "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps, "warmup": args.warmup,
+            "ms_per_step": ms, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+            "dtype": "mxfp4", "data": "synthetic",
+            "config": {"workload": args.config, "layers": {l.name: [l.b, l.n, l.m] for l in layers}, "g": g, "rounding": "SR",
+                       "out_dtype": "bf16", "flops_per_step": flops_step, "l2": "inputs_exceed_l2",
+                       "frac_of_4x_bf16_sustained": value / world / fp4_peak, "frac_of_nominal_9pf": value / world / NOMINAL_FP4_TFLOPS,
+                       "step_as_separate_calls_ms": calls_ms},
+            "e2e": {"value": e2e_value, "unit": UNIT, "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h, "ms_per_step": ms_e2e},
+            "gpu_launches": args.steps * len(layers) * 6,
+            "clocks": clocks,
+            "roofline": None if gemm_tflops is None else {
+                         "kernel": "gemm_mxf4_kernel", "bound": "tensor", "achieved": gemm_tflops, "peak": fp4_peak, "unit": "TFLOP/s",
+                         "frac": gemm_tflops / fp4_peak, "traffic": None,
+                         "peak_source": f"4 x {peaks['source']} sustained bf16 ({peaks['bf16_sustained']} TFLOP/s); no FP4 peak was measured"},
+            "kernels": kernels,
+            "hbm_peak_gbs": peaks["hbm_gbs"], "peaks_source": peaks["source"],
+            "cpu_baseline": cpu_baseline,
+        }))
+    if world > 1:
+        dist.destroy_process_group()
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=40)
+    ap.add_argument("--warmup", type=int, default=3)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--config", default="gpt_6p7b")
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--legs", default="value,roofline,e2e", help="comma list of GPU legs to run (profiling runs use 'value')")
+    args = ap.parse_args()
+    if args.impl == "reference":
+        run_reference(args)
+    else:
+        run_gpu(args)
+
+
+if __name__ == "__main__":
+    main()

@@ -240,9 +240,22 @@ ORC_API uint32_t orc_rn_round(double w)
 /* Algorithm 1 (rounding = 1, RN) or Algorithm 2 (rounding = 0, SR) applied to
  * every 32 consecutive entries of each row of y [R, K] (fp32 pre-quantisation
  * values).  codes: one 4-bit code per byte [R, K]; scales: E8M0 [R, K/32]. */
+ORC_API int orc_quantize_rows(const float *y, int64_t R, int64_t K, int rounding,
+                              uint64_t seed, uint32_t stream_tag, const int64_t *row_ids,
+                              uint8_t *codes, uint8_t *scales);
+
 ORC_API int orc_quantize(const float *y, int64_t R, int64_t K, int rounding,
                          uint64_t seed, uint32_t stream_tag,
                          uint8_t *codes, uint8_t *scales)
+{
+    return orc_quantize_rows(y, R, K, rounding, seed, stream_tag, NULL, codes, scales);
+}
+
+/* Same, for a subset of the rows of a larger operand: row_ids[r] is the row index in the full K-major
+ * operand (it only enters through the element index that keys the SR draw); NULL = 0..R-1. */
+ORC_API int orc_quantize_rows(const float *y, int64_t R, int64_t K, int rounding,
+                              uint64_t seed, uint32_t stream_tag, const int64_t *row_ids,
+                              uint8_t *codes, uint8_t *scales)
 {
     if (K % 32 != 0) return -1;
     const int64_t nblk = K / 32;
@@ -263,9 +276,10 @@ ORC_API int orc_quantize(const float *y, int64_t R, int64_t K, int rounding,
             int shared_exp = (int)byte - 127;
             for (int i = 0; i < 32; ++i) {
                 int64_t idx = r * K + b * 32 + i;
+                int64_t elem = (row_ids ? row_ids[r] : r) * K + b * 32 + i;   /* index in the full operand */
                 if (rounding == 0) {
                     double w = ldexp(0.75 * (double)V[i], -shared_exp);   /* (3/4) V_i / X, exact */
-                    codes[idx] = (uint8_t)orc_sr_round(w, orc_sr_draw(seed, stream_tag, (uint64_t)idx));
+                    codes[idx] = (uint8_t)orc_sr_round(w, orc_sr_draw(seed, stream_tag, (uint64_t)elem));
                 } else {
                     double w = ldexp((double)V[i], -shared_exp);          /* V_i / X, exact */
                     codes[idx] = (uint8_t)orc_rn_round(w);

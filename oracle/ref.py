@@ -40,6 +40,8 @@ _lib.orc_rn_round.argtypes = [C.c_double]
 _lib.orc_rn_round.restype = C.c_uint32
 _lib.orc_quantize.argtypes = [_f32p, _i64, _i64, C.c_int, _u64, C.c_uint32, _u8p, _u8p]
 _lib.orc_quantize.restype = C.c_int
+_lib.orc_quantize_rows.argtypes = [_f32p, _i64, _i64, C.c_int, _u64, C.c_uint32, C.c_void_p, _u8p, _u8p]
+_lib.orc_quantize_rows.restype = C.c_int
 _lib.orc_pack.argtypes = [_u8p, _i64, _u8p]
 _lib.orc_pack.restype = None
 _lib.orc_dequantize.argtypes = [_u8p, _u8p, _i64, _i64, _f64p]
@@ -122,20 +124,23 @@ def rht(x: np.ndarray, g: int, seed: int, transpose: bool = False) -> np.ndarray
     return y
 
 
-def quantize(y: np.ndarray, rounding: int, seed: int, stream_tag: int):
-    """fp32 pre-quantisation values [R, K] -> (codes [R, K] one per byte, scales [R, K/32])."""
+def quantize(y: np.ndarray, rounding: int, seed: int, stream_tag: int, row_ids=None):
+    """fp32 pre-quantisation values [R, K] -> (codes [R, K] one per byte, scales [R, K/32]).
+
+    row_ids: when y holds a subset of the rows of a larger operand, their row indices there (they key the SR draws)."""
     y = np.ascontiguousarray(y, np.float32)
     R, K = y.shape
     codes = np.empty((R, K), np.uint8)
     scales = np.empty((R, K // 32), np.uint8)
-    if _lib.orc_quantize(y, R, K, rounding, seed, stream_tag, codes, scales) != 0:
+    rp, _n, _keep = _idx(row_ids)
+    if _lib.orc_quantize_rows(y, R, K, rounding, seed, stream_tag, rp, codes, scales) != 0:
         raise ValueError("K must be a multiple of 32")
     return codes, scales
 
 
-def rht_quantize(x, g, rounding, seed, stream_tag, transpose=False):
+def rht_quantize(x, g, rounding, seed, stream_tag, transpose=False, row_ids=None):
     y = rht(x, g, seed, transpose)
-    codes, scales = quantize(y, rounding, seed, stream_tag)
+    codes, scales = quantize(y, rounding, seed, stream_tag, row_ids)
     return y, codes, scales
 
 

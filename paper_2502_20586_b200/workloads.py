@@ -107,6 +107,37 @@ def layer_inputs(config: str, layer: Linear, seed: int = 0):
     return dY, X, W
 
 
+def layer_inputs_device(config: str, layer: Linear, seed: int = 0, device="cuda"):
+    """Same distributions as layer_inputs, drawn on the GPU with torch's seeded generator (the full-size
+    tensors have up to 2.7e8 entries; numpy would take minutes).  Returns bf16 torch tensors (dY, X, W)."""
+    import torch
+    cid = CONFIG_IDS[config]
+    lid = [l.name for l in CONFIGS[config][0]].index(layer.name)
+    gen = torch.Generator(device=device)
+    gen.manual_seed(1_000_003 * seed + 1009 * cid + lid)
+
+    def normal(shape):
+        return torch.randn(shape, generator=gen, device=device, dtype=torch.float32)
+
+    def student_t3(shape):
+        chi2 = normal(shape).square_()
+        chi2 += normal(shape).square_()
+        chi2 += normal(shape).square_()
+        return normal(shape).div_(chi2.div_(3.0).sqrt_())
+
+    std = 1e-3 if config == "single_256x512" else 1e-4
+    dY = student_t3((layer.b, layer.m)).mul_(std / 3.0 ** 0.5)
+    if config == "single_256x512":
+        mask = torch.rand((layer.b, layer.m), generator=gen, device=device) < 1e-3
+        dY = torch.where(mask, dY * 50.0, dY)
+    X = normal((layer.b, layer.n))
+    if config != "single_256x512":
+        cols = torch.randperm(layer.n, generator=gen, device=device)[:8]
+        X[:, cols] *= 20.0
+    W = normal((layer.m, layer.n)).mul_(0.02)
+    return dY.to(torch.bfloat16), X.to(torch.bfloat16), W.to(torch.bfloat16)
+
+
 def ablation_inputs(M: int, N: int, K: int, outlier_rate: float, seed: int = 0):
     """One GEMM C = A B^T with a gradient-like A [M, K] and a weight-like B [N, K]."""
     ra, rb = _rng(seed, 100, 0), _rng(seed, 100, 1)
