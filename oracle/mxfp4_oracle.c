@@ -28,8 +28,10 @@
  *   - shared_exp = floor(log2 amax) - 2, clamped to [-127, 127]; an all-zero
  *     block takes -127.  The scale byte is OCP E8M0: byte = shared_exp + 127.
  *   - SR acts on the exact real w = (3/4) V_i / X; with f <= |w| < c the grid
- *     neighbours, round up iff  r + 1/2 < 256 (|w| - f)/(c - f),  r a uniform
- *     8-bit integer from Philox4x32-10 keyed on (seed, element index).
+ *     neighbours and frac = (|w| - f)/(c - f), round up iff
+ *     frac >= (r + 1/2)/256,  r a uniform 8-bit integer from Philox4x32-10
+ *     keyed on (seed, element index).  This is Eq. 2 with the dither
+ *     delta = 1/2 - (r + 1/2)/256 in (-1/2, 1/2): ceil iff x + delta >= floor(x) + 1/2.
  *   - RN is round-to-nearest, ties to the code with even mantissa bit,
  *     saturating at 6.
  *   - The sign bit of the input is kept (a negative value may round to -0).
@@ -205,7 +207,8 @@ ORC_API uint32_t orc_e8m0_from_amax(float amax)
 }
 
 /* stochastic_round_to_FP4 (Algorithm 2 line 5) on the exact real w, |w| <= 6:
- * f <= |w| < c neighbours on the enumerated grid; up iff r + 1/2 < 256 frac. */
+ * f <= |w| < c neighbours on the enumerated grid; Eq. 2 in units of the local
+ * grid step with delta = 1/2 - (r + 1/2)/256: up iff frac + delta >= 1/2. */
 ORC_API uint32_t orc_sr_round(double w, uint32_t r)
 {
     uint32_t sign = signbit(w) ? 8u : 0u;
@@ -215,7 +218,7 @@ ORC_API uint32_t orc_sr_round(double w, uint32_t r)
     while (lo + 1 < 8 && E2M1_GRID[lo + 1] <= a) ++lo;    /* f = grid[lo] <= a < grid[lo+1] = c */
     double f = E2M1_GRID[lo], c = E2M1_GRID[lo + 1];
     double frac = (a - f) / (c - f);
-    int up = ((double)r + 0.5) < frac * 256.0;
+    int up = frac * 256.0 >= ((double)r + 0.5);
     return sign | (lo + (uint32_t)up);
 }
 

@@ -223,13 +223,14 @@ def test_sr_is_unbiased_by_enumeration(ref):
 def test_sr_matches_dither_form_on_uniform_grid(ref):
     """Eq. 1-2 on the uniform part of the grid (spacing 1/2 on [0, 2]): delta = 1/2 - (r + 1/2)/256."""
     rng = np.random.default_rng(2)
-    for w in rng.uniform(0, 2, 400):
+    ties = [(k + 0.5) / 512 for k in (0, 1, 77, 128, 200, 255, 256, 300, 511, 767, 1023)]   # frac * 256 = r + 1/2 exactly
+    for w in list(rng.uniform(0, 2, 400)) + ties:
         x = 2 * w                                              # grid-index units: integers are grid points
         for r in (0, 1, 77, 128, 200, 255):
             delta = 0.5 - (r + 0.5) / 256.0
-            if abs((x - np.floor(x)) * 256 - (r + 0.5)) < 1e-9:
-                continue                                       # the measure-zero tie
-            expect = np.ceil(x) if x + delta >= np.floor(x) + 0.5 else np.floor(x)
+            expect = np.ceil(x) if (x - np.floor(x)) + delta >= 0.5 else np.floor(x)
+            if x == np.floor(x):
+                expect = x
             assert ref.e2m1_value(ref.sr_round(w, r)) == expect / 2
 
 
