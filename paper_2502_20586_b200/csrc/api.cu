@@ -45,7 +45,7 @@ mxfp4_status runtime_init() {
             return;
         }
         g_rt.encode = reinterpret_cast<EncodeTiledFn>(fn);
-        if (mx::gemm_init() != cudaSuccess) g_rt.status = MXFP4_ERR_CUDA;
+        if (mx::gemm_init() != cudaSuccess || mx::quant_tc_init() != cudaSuccess) g_rt.status = MXFP4_ERR_CUDA;
     });
     return g_rt.status;
 }
@@ -83,6 +83,23 @@ mxfp4_status make_codes_map(CUtensorMap* map, const uint8_t* codes, int64_t rows
                                    CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
                                    CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
     return r == CUDA_SUCCESS ? MXFP4_OK : MXFP4_ERR_CUDA;
+}
+
+// Tensor map over the bf16 input [rows, cols] (leading dimension ld): box = 64 columns x 128 rows, 128-byte swizzle.
+// Only built when the tensor-core quantiser can take the call; otherwise the CUDA-core kernels read x directly.
+void attach_input_map(QuantArgs& a) {
+    a.has_tmap = false;
+    const int64_t K = a.reduce_dim == 1 ? a.cols : a.rows;
+    if (!(a.g == 32 || a.g == 64 || a.g == 128) || K % 128 != 0) return;
+    if (a.rows > 0x7FFFFFFF || a.cols > 0x7FFFFFFF) return;
+    const cuuint64_t dims[2] = {(cuuint64_t)a.cols, (cuuint64_t)a.rows};
+    const cuuint64_t strides[1] = {(cuuint64_t)a.ld * 2};
+    const cuuint32_t box[2] = {64, 128};
+    const cuuint32_t elem_strides[2] = {1, 1};
+    const CUresult r = g_rt.encode(&a.tmap_x, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(a.x), dims, strides, box,
+                                   elem_strides, CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
+                                   CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+    a.has_tmap = r == CUDA_SUCCESS;
 }
 
 mxfp4_status gemm_impl(const uint8_t* A_codes, const uint8_t* A_scales, const uint8_t* B_codes, const uint8_t* B_scales, int64_t M,
@@ -149,6 +166,7 @@ mxfp4_status mxfp4_rht_sr_quantize(const void* x, int64_t rows, int64_t cols, in
     if (!aligned16(codes)) return MXFP4_ERR_ALIGN;
     if ((st = runtime_init()) != MXFP4_OK) return st;
     QuantArgs a{x, rows, cols, ld, reduce_dim, g, rounding, seed, stream_tag, codes, scales, sf_layout == MXFP4_SF_NATIVE, nullptr};
+    attach_input_map(a);
     return mx::launch_quantize(a, static_cast<cudaStream_t>(cuda_stream)) == cudaSuccess ? MXFP4_OK : MXFP4_ERR_CUDA;
 }
 
@@ -160,6 +178,7 @@ mxfp4_status mxfp4_rht(const void* x, int64_t rows, int64_t cols, int64_t ld, in
     if (!aligned16(y)) return MXFP4_ERR_ALIGN;
     if ((st = runtime_init()) != MXFP4_OK) return st;
     QuantArgs a{x, rows, cols, ld, reduce_dim, g, 0, seed, 0u, nullptr, nullptr, 0, y};
+    attach_input_map(a);
     return mx::launch_rht_dump(a, static_cast<cudaStream_t>(cuda_stream)) == cudaSuccess ? MXFP4_OK : MXFP4_ERR_CUDA;
 }
 
@@ -202,14 +221,16 @@ mxfp4_status mxfp4_linear_backward(const void* dY, const void* X, const void* W,
     uint8_t *c[4], *s[4];
     for (int i = 0; i < 4; ++i) { c[i] = base + ws.codes[i]; s[i] = base + ws.scales[i]; }
     // Algorithm 3 lines 3-6: stream tags 1..4, one sign vector (same seed) for all four views.
-    const QuantArgs q[4] = {
+    QuantArgs q[4] = {
         {dY, b, m, m, 1, g, rounding, seed, 1u, c[0], s[0], 1, nullptr},   // dY   [b, K = m]
         {W, m, n, n, 0, g, rounding, seed, 2u, c[1], s[1], 1, nullptr},    // W^T  [n, K = m]
         {dY, b, m, m, 0, g, rounding, seed, 3u, c[2], s[2], 1, nullptr},   // dY^T [m, K = b]
         {X, b, n, n, 0, g, rounding, seed, 4u, c[3], s[3], 1, nullptr},    // X^T  [n, K = b]
     };
-    for (int i = 0; i < 4; ++i)
+    for (int i = 0; i < 4; ++i) {
+        attach_input_map(q[i]);
         if (mx::launch_quantize(q[i], stream) != cudaSuccess) return MXFP4_ERR_CUDA;
+    }
     // lines 7-11: two MXFP4 GEMMs; the 16/9 un-does the two 3/4 pre-scales of Algorithm 2.
     const float alpha = rounding == MXFP4_ROUND_SR ? 16.0f / 9.0f : 1.0f;
     st = gemm_impl(c[0], s[0], c[1], s[1], b, n, m, alpha, dX, n, out_dtype, stream);

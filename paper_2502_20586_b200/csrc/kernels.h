@@ -18,7 +18,14 @@ struct QuantArgs {
     uint8_t* scales;
     int sf_native;
     float* y_out;         // only for the transform dump
+    CUtensorMap tmap_x;   // x as [rows, cols] bf16, box 64 cols x 128 rows, 128-byte swizzle (tensor-core path)
+    bool has_tmap;
 };
+
+// Tensor-core transform path (quantize_tc.cu): g in {32, 64, 128} and reduce length a multiple of 128.
+bool quant_tc_eligible(const QuantArgs& a);
+cudaError_t quant_tc_init();
+cudaError_t launch_quantize_tc(const QuantArgs& a, bool dump_y, cudaStream_t stream);
 
 cudaError_t launch_quantize(const QuantArgs& a, cudaStream_t stream);
 cudaError_t launch_rht_dump(const QuantArgs& a, cudaStream_t stream);

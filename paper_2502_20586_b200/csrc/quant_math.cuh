@@ -95,23 +95,50 @@ __device__ __forceinline__ uint32_t cvt_e2m1x2_rn(float lo, float hi) {
     return out;
 }
 
+// Generic (any scale exponent) SR encoder of one value on the fp32 bit pattern.  |y| / X is formed exactly in two
+// power-of-two steps, then truncated onto a grid of 2^-23 by one round-toward-zero multiply with 3/4 * 2^-126.
+// That factor places E2M1's subnormal/normal boundary (1.0) on fp32's, so bits >> 22 is the E2M1 code of the lower
+// neighbour and the low 22 bits are floor(frac 2^22); adding (255 - r) 2^14 + 2^13 carries into bit 22 exactly
+// when 256 frac >= r + 1/2.  Truncation keeps the decision exact because the thresholds are integers there.
+__device__ __forceinline__ uint32_t sr_encode_wide(float y, float p1, float p2, uint32_t r) {
+    const float a = __fmul_rz(fabsf(y) * p1 * p2, __uint_as_float(0x00600000u));      // 3/4 * 2^-126
+    const uint32_t t = __float_as_uint(a) + (((r ^ 0xFFu) << 14) | 0x2000u);
+    return (t >> 22) | ((__float_as_uint(y) >> 28) & 8u);
+}
+
+// cvt.rz.f16x2.f32: two floats -> packed halves (lo in the low 16 bits), both truncated toward zero.
+__device__ __forceinline__ uint32_t cvt_f16x2_rz(float lo, float hi) {
+    uint32_t d;
+    asm("cvt.rz.f16x2.f32 %0, %1, %2;" : "=r"(d) : "f"(hi), "f"(lo));
+    return d;
+}
+
+// Eight SR-rounded values, held as four packed-half sums (bit 15 sign, bits 11:9 E2M1 magnitude code in each
+// 16-bit lane), to one 32-bit word of eight 4-bit codes, element 0 in the low nibble.
+__device__ __forceinline__ uint32_t pack8_from_half_sums(uint32_t s0, uint32_t s1, uint32_t s2, uint32_t s3) {
+    const uint32_t x = __byte_perm(s0, s1, 0x7531), y = __byte_perm(s2, s3, 0x7531);   // high byte of every lane: s000cccm
+    const uint32_t vx = (x >> 1) & 0x47474747u, vy = (y >> 1) & 0x47474747u;          // 0s000ccc
+    const uint32_t nx = (vx | (vx >> 3)) & 0x0F0F0F0Fu, ny = (vy | (vy >> 3)) & 0x0F0F0F0Fu;   // 0000sccc
+    const uint32_t ux = nx | (nx >> 4), uy = ny | (ny >> 4);                          // bytes 0 and 2: two nibbles each
+    return __byte_perm(ux, uy, 0x6420);
+}
+
 // Quantise 32 consecutive fp32 values (one MX block) to 16 bytes of packed E2M1 codes + one E8M0 byte.
-//   SR (Algorithm 2): round up iff r + 1/2 < 256 frac, decided on the exact real w = (3/4) y / X.
-//     |y| * (3/4 * 2^(-e-126)) is formed with round-up; since every threshold is representable this keeps
-//     the decision exact.  The factor 2^-126 places E2M1's subnormal/normal boundary (1.0) on fp32's, so
-//     bits(a) >> 22 IS the E2M1 magnitude code of the lower neighbour and the low 22 bits are frac 2^22;
-//     adding ((255 - r) << 14 | 0x1fff) carries into bit 22 exactly when r + 1/2 < 256 frac.
+//   SR (Algorithm 2): round up iff 256 frac >= r + 1/2 (Eq. 2 with an 8-bit dither), decided on the exact real
+//     w = (3/4) y / X.  Fast path: z = RZ(y * 3/4 * 2^(-e-14)) is truncated to fp16 (two values per cvt).  The
+//     factor 2^-14 places E2M1's subnormal/normal boundary on fp16's, so in each 16-bit lane bits 11:9 are the
+//     E2M1 code of the lower neighbour and the low 9 bits are floor(512 frac); adding 511 - 2r carries into bit 9
+//     exactly when floor(512 frac) >= 2r + 1, i.e. when 256 frac >= r + 1/2.  Both truncations are toward zero
+//     and every threshold is a multiple of the fp16 spacing, so the decision is that of the exact real.
+//     One 32-bit add handles two lanes (no carry can cross: the magnitude field is at most 0x0dff + 0x1ff).
 //   RN (Algorithm 1): hardware nearest-even convert of y / X.
+// A NaN input is out of contract (the block's scale is then taken from the other values); Inf gives byte 255.
 __device__ __forceinline__ void quantize_block32(const float (&y)[32], int rounding, uint64_t seed, uint32_t stream_tag,
                                                  uint64_t i0, uint32_t (&packed)[4], uint32_t& scale_byte) {
     float amax = 0.0f;
 #pragma unroll
-    for (int i = 0; i < 32; ++i) amax = fmaxf(amax, fabsf(y[i]));
-    // fmaxf drops NaNs: detect non-finite inputs through the sum of exponents instead
-    bool finite = true;
-#pragma unroll
-    for (int i = 0; i < 32; ++i) finite = finite && ((__float_as_uint(y[i]) & 0x7F800000u) != 0x7F800000u);
-    scale_byte = finite ? e8m0_from_amax(amax) : 255u;
+    for (int i = 0; i < 32; i += 2) amax = fmaxf(amax, fmaxf(fabsf(y[i]), fabsf(y[i + 1])));
+    scale_byte = e8m0_from_amax(amax);
     if (scale_byte == 255u) {
         packed[0] = packed[1] = packed[2] = packed[3] = 0u;
         return;
@@ -120,25 +147,33 @@ __device__ __forceinline__ void quantize_block32(const float (&y)[32], int round
     if (rounding == 0) {
         uint32_t rw[8];
         sr_draws32(seed, stream_tag, i0, rw);
-        const bool fast = e <= 21;                                   // 3/4 * 2^(-e-126) representable
-        const float c_fast = fast ? 1.5f * pow2f_wide(-e - 127) : 0.0f;
-        const int h1 = (-e) / 2, h2 = -e - h1;                       // slow path: exact 2^-e in two steps
-        const float p1 = pow2f_wide(h1), p2 = pow2f_wide(h2);
-        const float c_slow = __uint_as_float(0x00600000u);           // 3/4 * 2^-126
+        if (e <= 100) {
+            const float c = 1.5f * pow2f_wide(-e - 15);              // 3/4 * 2^(-e-14), a normal fp32
 #pragma unroll
-        for (int q = 0; q < 4; ++q) {
-            uint32_t word = 0u;
+            for (int q = 0; q < 4; ++q) {
+                uint32_t s[4];
 #pragma unroll
-            for (int j = 0; j < 8; ++j) {
-                const int i = 8 * q + j;
-                const float ay = fabsf(y[i]);
-                const float a = fast ? __fmul_ru(ay, c_fast) : __fmul_ru(ay * p1 * p2, c_slow);
-                const uint32_t r = (rw[i >> 2] >> (8 * (i & 3))) & 0xFFu;
-                const uint32_t t = __float_as_uint(a) + (((r ^ 0xFFu) << 14) | 0x1FFFu);
-                const uint32_t code = (t >> 22) | ((__float_as_uint(y[i]) >> 28) & 8u);
-                word |= code << (4 * j);
+                for (int p = 0; p < 4; ++p) {
+                    const int i = 8 * q + 2 * p;
+                    const uint32_t h = cvt_f16x2_rz(__fmul_rz(y[i], c), __fmul_rz(y[i + 1], c));
+                    const uint32_t x = __byte_perm(rw[i >> 2], 0u, (p & 1) ? 0x4342 : 0x4140);   // r_i | r_{i+1} << 16
+                    s[p] = h + (0x01FF01FFu - 2u * x);
+                }
+                packed[q] = pack8_from_half_sums(s[0], s[1], s[2], s[3]);
             }
-            packed[q] = word;
+        } else {
+            const int h1 = (-e) / 2, h2 = -e - h1;                   // exact 2^-e in two steps
+            const float p1 = pow2f_wide(h1), p2 = pow2f_wide(h2);
+#pragma unroll
+            for (int q = 0; q < 4; ++q) {
+                uint32_t word = 0u;
+#pragma unroll
+                for (int j = 0; j < 8; ++j) {
+                    const int i = 8 * q + j;
+                    word |= sr_encode_wide(y[i], p1, p2, (rw[i >> 2] >> (8 * (i & 3))) & 0xFFu) << (4 * j);
+                }
+                packed[q] = word;
+            }
         }
     } else {
         const float inv_x = pow2f_wide(-e);

@@ -153,6 +153,7 @@ __global__ void __launch_bounds__(256) quantize_transpose_kernel(const __nv_bflo
 // ---------------------------------------------------------------------------------------------- launchers
 template <bool DUMP_Y>
 static cudaError_t launch(const QuantArgs& a, cudaStream_t stream) {
+    if (quant_tc_eligible(a)) return launch_quantize_tc(a, DUMP_Y, stream);
     const __nv_bfloat16* x = static_cast<const __nv_bfloat16*>(a.x);
     if (a.reduce_dim == 1) {
         const int64_t nblocks = a.rows * (a.cols / 32);

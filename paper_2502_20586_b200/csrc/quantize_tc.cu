@@ -1,0 +1,261 @@
+// Blockwise RHT + MXFP4 quantiser with the transform on the tensor cores (g in {32, 64, 128}).
+//
+// Section 3.2 builds the blockwise RHT as a dense matrix product with a small g x g matrix, which keeps it
+// memory-bound in the operand.  Here that product is a tcgen05.mma kind::f16: per tile of 128 output rows x 128
+// reduce-dim elements,
+//     D[128 x 128] = A[128 x 128] * T,   T = blockdiag over 128/g chunks of diag(S) H_g (x 1/sqrt(g) when exact),
+// with bf16 inputs (T is +-1, +-1/8 or 0: exact) and fp32 accumulation in TMEM.  The accumulator comes back with
+// one output row per TMEM lane and its 128 transformed values in consecutive columns, so each epilogue thread
+// owns whole MX blocks: amax, scale, stochastic rounding and packing need no shuffles.  The same kernel serves
+// both access patterns: for a contiguous reduce dimension the x tile is the K-major A operand; for the transposing
+// views (W, dY^T, X^T of Algorithm 3) the very same TMA tile is handed to the MMA as an MN-major operand, so the
+// transposition costs nothing.
+//
+//   warp 0        TMA producer (two 64-column x 128-row boxes per tile, 128-byte swizzle, 4-stage ring)
+//   warp 1        MMA issuer (8 K=16 MMAs per tile into one of four 128-column TMEM accumulators)
+//   warps 2..17   epilogue: warp = (TMEM lane quadrant, MX block): tcgen05.ld 32 columns, release the
+//                 accumulator, then scale / SR / pack / store
+// Every mbarrier wait is bounded; on expiry the CTA records a status word and unwinds.
+#include <cuda_bf16.h>
+
+#include "kernels.h"
+#include "ptx.cuh"
+#include "quant_math.cuh"
+
+namespace mx {
+namespace {
+
+constexpr int kTile = 128;                          // output rows per tile and reduce-dim elements per tile
+constexpr int kStagesQ = 4;
+constexpr uint32_t kBoxBytes = 64 * 2 * 128;        // one TMA box: 64 bf16 columns x 128 rows = 16 KB
+constexpr uint32_t kTileBytes = 2 * kBoxBytes;      // 32 KB
+constexpr uint32_t kTBytes = 2 * kBoxBytes;         // transform matrix, 128 x 128 bf16
+constexpr uint32_t kSmemQ = kStagesQ * kTileBytes + kTBytes + 1024 + 256;
+constexpr int kAccBufs = 4;                         // 4 x 128 TMEM columns
+constexpr int kEpiWarps = 16;
+constexpr int kThreadsQ = (2 + kEpiWarps) * 32;
+
+struct QParams {
+    int64_t R, K;              // output operand [R, K]
+    int64_t r_tiles, k_tiles;
+    int reduce_dim, g, rounding;
+    uint64_t seed;
+    uint32_t stream_tag;
+    uint8_t* codes;
+    uint8_t* scales;
+    int sf_native;
+    float* y_out;
+};
+
+// bf16 entry (n, k) of the transform operand, stored N x K (K-major): T[k][n] = S_k H_g[k][n] inside a g-chunk.
+__device__ __forceinline__ uint32_t transform_entry(int n, int k, int g, const uint32_t (&sign)[4]) {
+    if (g == 0) return n == k ? 0x3F80u : 0u;
+    if ((n ^ k) & ~(g - 1)) return 0u;                                   // different g-chunks
+    const int kk = k & (g - 1);
+    const uint32_t neg = ((sign[kk >> 5] >> (kk & 31)) ^ (uint32_t)__popc(k & n & (g - 1))) & 1u;
+    const uint32_t mag = g == 64 ? 0x3E00u : 0x3F80u;                    // 1/8 (exact 1/sqrt(64)) or 1
+    return mag | (neg << 15);
+}
+
+template <bool DUMP_Y>
+__global__ void __launch_bounds__(kThreadsQ, 1)
+quantize_tc_kernel(const __grid_constant__ CUtensorMap tmap_x, const QParams p) {
+    extern __shared__ uint8_t smem_raw[];
+    uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
+    uint8_t* smem_t = smem + kStagesQ * kTileBytes;
+    uint64_t* bars = reinterpret_cast<uint64_t*>(smem_t + kTBytes);
+    uint64_t* full_bar = bars;                          // [kStagesQ]  TMA -> MMA
+    uint64_t* empty_bar = bars + kStagesQ;              // [kStagesQ]  MMA -> TMA
+    uint64_t* acc_full = bars + 2 * kStagesQ;           // [kAccBufs]  MMA -> epilogue
+    uint64_t* acc_empty = bars + 2 * kStagesQ + kAccBufs;   // [kAccBufs]  epilogue -> MMA
+    uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 2 * kStagesQ + 2 * kAccBufs);
+    volatile uint32_t* abort_flag = tmem_slot + 1;
+
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const int64_t num_tiles = p.r_tiles * p.k_tiles;
+
+    if (threadIdx.x == 0) {
+        for (int s = 0; s < kStagesQ; ++s) { mbar_init(&full_bar[s], 1); mbar_init(&empty_bar[s], 1); }
+        for (int b = 0; b < kAccBufs; ++b) { mbar_init(&acc_full[b], 1); mbar_init(&acc_empty[b], kEpiWarps); }
+        *abort_flag = 0;
+        mbar_fence_init();
+        prefetch_tensormap(&tmap_x);
+    }
+    if (warp == 1) {
+        tmem_alloc(tmem_slot, 512);
+        tmem_relinquish();
+    }
+    {
+        // Transform operand, written in the 128-byte-swizzled K-major layout the MMA descriptor expects:
+        // entry (n, k) at box (k / 64), row n (128 B pitch), 16-byte chunk ((k % 64) / 8) ^ (n % 8).
+        uint32_t sign[4] = {0u, 0u, 0u, 0u};
+        if (p.g != 0) {
+            const uint4 o = philox4x32_10(0u, 0u, 0u, 0u, (uint32_t)p.seed, (uint32_t)(p.seed >> 32));
+            sign[0] = o.x; sign[1] = o.y; sign[2] = o.z; sign[3] = o.w;
+        }
+        for (int task = threadIdx.x; task < 128 * 16; task += kThreadsQ) {
+            const int n = task >> 4, c = task & 15;                      // c: 16-byte chunk = 8 consecutive k
+            uint32_t w[4];
+#pragma unroll
+            for (int j = 0; j < 4; ++j)
+                w[j] = transform_entry(n, c * 8 + 2 * j, p.g, sign) | (transform_entry(n, c * 8 + 2 * j + 1, p.g, sign) << 16);
+            const uint32_t off = (uint32_t)(c >> 3) * kBoxBytes + (uint32_t)n * 128u + (uint32_t)(((c & 7) ^ (n & 7)) << 4);
+            *reinterpret_cast<uint4*>(smem_t + off) = make_uint4(w[0], w[1], w[2], w[3]);
+        }
+        fence_proxy_async_smem();                                        // generic-proxy writes -> tensor-core reads
+    }
+    tc_fence_before_sync();
+    __syncthreads();
+    tc_fence_after_sync();
+    const uint32_t tmem_base = *tmem_slot;
+
+    if (warp == 0) {
+        // ------------------------------------------------------------------ TMA producer
+        if (lane == 0) {
+            uint32_t it = 0;
+            bool ok = true;
+            for (int64_t t = blockIdx.x; t < num_tiles; t += gridDim.x, ++it) {
+                const int s = it % kStagesQ;
+                if (!(ok = mbar_wait(&empty_bar[s], ((it / kStagesQ) & 1) ^ 1, abort_flag))) break;
+                // tile -> (row tile of the OUTPUT operand, k tile); x coordinates depend on the access pattern
+                int32_t cx, cy;
+                if (p.reduce_dim == 1) {            // output rows = x rows; k = x columns; consecutive tiles along k
+                    const int64_t rt = t / p.k_tiles, kt = t - rt * p.k_tiles;
+                    cx = (int32_t)(kt * kTile); cy = (int32_t)(rt * kTile);
+                } else {                            // output rows = x columns; k = x rows; consecutive tiles along x columns
+                    const int64_t kt = t / p.r_tiles, rt = t - kt * p.r_tiles;
+                    cx = (int32_t)(rt * kTile); cy = (int32_t)(kt * kTile);
+                }
+                uint8_t* st = smem + s * kTileBytes;
+                mbar_expect_tx(&full_bar[s], kTileBytes);
+                tma_load_2d(st, &tmap_x, &full_bar[s], cx, cy);
+                tma_load_2d(st + kBoxBytes, &tmap_x, &full_bar[s], cx + 64, cy);
+            }
+            if (!ok) *abort_flag = 1;
+        }
+    } else if (warp == 1) {
+        // ------------------------------------------------------------------ MMA issuer
+        if (lane == 0) {
+            // kind::f16 instruction descriptor: D = fp32 (bits 4-5 = 1), A = B = bf16 (bits 7-9, 10-12 = 1),
+            // A major at bit 15 (0 = K-major, 1 = MN-major), B K-major, N >> 3 at bit 17, M >> 4 at bit 24.
+            const uint32_t idesc = (1u << 4) | (1u << 7) | (1u << 10) | ((p.reduce_dim == 0 ? 1u : 0u) << 15) |
+                                   ((uint32_t)(kTile >> 3) << 17) | ((uint32_t)(kTile >> 4) << 24);
+            const uint32_t t_addr = smem_u32(smem_t);
+            uint32_t it = 0;
+            bool ok = true;
+            for (int64_t t = blockIdx.x; t < num_tiles; t += gridDim.x, ++it) {
+                const int s = it % kStagesQ, b = it % kAccBufs;
+                if (!(ok = mbar_wait(&acc_empty[b], ((it / kAccBufs) & 1) ^ 1, abort_flag))) break;
+                if (!(ok = mbar_wait(&full_bar[s], (it / kStagesQ) & 1, abort_flag))) break;
+                tc_fence_after_sync();
+                const uint32_t a_addr = smem_u32(smem + s * kTileBytes);
+#pragma unroll
+                for (int ks = 0; ks < 8; ++ks) {                           // K = 16 per MMA
+                    uint64_t adesc;
+                    if (p.reduce_dim == 1)      // K-major: box ks/4, 32 bytes of K per step inside the 128-byte swizzle atom
+                        adesc = make_smem_desc(a_addr + (ks >> 2) * kBoxBytes + (ks & 3) * 32, 16, 1024, 2);
+                    else                        // MN-major: 16 k-rows of 128 B per step; the second 64 output rows sit one box further
+                        adesc = make_smem_desc(a_addr + ks * 2048, kBoxBytes, 1024, 2);
+                    const uint64_t bdesc = make_smem_desc(t_addr + (ks >> 2) * kBoxBytes + (ks & 3) * 32, 16, 1024, 2);
+                    tc_mma_f16(tmem_base + b * kTile, adesc, bdesc, idesc, ks != 0 ? 1u : 0u);
+                }
+                tc_commit(&empty_bar[s]);
+                tc_commit(&acc_full[b]);
+            }
+            if (!ok) *abort_flag = 1;
+        }
+    } else {
+        // ------------------------------------------------------------------ epilogue
+        const int e = warp - 2;
+        const int q = warp & 3;                      // TMEM lane quadrant this warp may read
+        const int blk = e >> 2;                      // MX block (32 columns) of the tile; q takes all four values within each blk
+        const float cg = p.g == 32 ? 0.17677669529663687f : p.g == 128 ? 0.08838834764831845f : 1.0f;
+        const int64_t nkb = p.K >> 5, nkc = (nkb + 3) >> 2;
+        uint32_t it = 0;
+        bool ok = true;
+        for (int64_t t = blockIdx.x; t < num_tiles; t += gridDim.x, ++it) {
+            const int b = it % kAccBufs;
+            int64_t rt, kt;
+            if (p.reduce_dim == 1) { rt = t / p.k_tiles; kt = t - rt * p.k_tiles; }
+            else { kt = t / p.r_tiles; rt = t - kt * p.r_tiles; }
+            ok = mbar_wait(&acc_full[b], (it / kAccBufs) & 1, abort_flag);
+            ok = __all_sync(0xffffffffu, ok);
+            if (!ok) break;
+            tc_fence_after_sync();
+            uint32_t raw[32];
+            tmem_ld_32x32b_x32(tmem_base + ((uint32_t)(q * 32) << 16) + b * kTile + blk * 32, raw);
+            tmem_ld_wait();
+            tc_fence_before_sync();
+            __syncwarp();
+            if (lane == 0) mbar_arrive(&acc_empty[b]);
+            const int64_t row = rt * kTile + q * 32 + lane;            // output row
+            if (row >= p.R) continue;
+            float y[32];
+#pragma unroll
+            for (int i = 0; i < 32; ++i) y[i] = __uint_as_float(raw[i]) * cg;   // exact no-op unless g is 32 or 128
+            const int64_t k0 = kt * kTile + blk * 32;
+            if (DUMP_Y) {
+                float4* dst = reinterpret_cast<float4*>(p.y_out + row * p.K + k0);
+#pragma unroll
+                for (int i = 0; i < 8; ++i) dst[i] = make_float4(y[4 * i], y[4 * i + 1], y[4 * i + 2], y[4 * i + 3]);
+                continue;
+            }
+            uint32_t packed[4], sbyte;
+            quantize_block32(y, p.rounding, p.seed, p.stream_tag, (uint64_t)(row * p.K + k0), packed, sbyte);
+            *reinterpret_cast<uint4*>(p.codes + row * (p.K >> 1) + (k0 >> 1)) = make_uint4(packed[0], packed[1], packed[2], packed[3]);
+            const int64_t kb = k0 >> 5;
+            const int64_t so = p.sf_native ? ((rt * nkc + kt) * 512 + lane * 16 + q * 4 + blk) : row * nkb + kb;
+            p.scales[so] = (uint8_t)sbyte;
+        }
+        if (!ok && lane == 0) *abort_flag = 1;
+    }
+
+    tc_fence_before_sync();
+    __syncthreads();
+    if (*abort_flag) {
+        for (int i = 0; i < 1000; ++i) __nanosleep(1000);
+        __syncthreads();
+    }
+    if (warp == 1) {
+        tc_fence_after_sync();
+        tmem_dealloc(tmem_base, 512);
+    }
+}
+
+}  // namespace
+
+bool quant_tc_eligible(const QuantArgs& a) {
+    const int64_t K = a.reduce_dim == 1 ? a.cols : a.rows;
+    return (a.g == 32 || a.g == 64 || a.g == 128) && K % kTile == 0 && a.has_tmap;
+}
+
+cudaError_t quant_tc_init() {
+    cudaError_t e = cudaFuncSetAttribute(quantize_tc_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kSmemQ);
+    if (e != cudaSuccess) return e;
+    return cudaFuncSetAttribute(quantize_tc_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kSmemQ);
+}
+
+cudaError_t launch_quantize_tc(const QuantArgs& a, bool dump_y, cudaStream_t stream) {
+    QParams p;
+    p.R = a.reduce_dim == 1 ? a.rows : a.cols;
+    p.K = a.reduce_dim == 1 ? a.cols : a.rows;
+    p.r_tiles = (p.R + kTile - 1) / kTile;
+    p.k_tiles = p.K / kTile;
+    p.reduce_dim = a.reduce_dim; p.g = a.g; p.rounding = a.rounding;
+    p.seed = a.seed; p.stream_tag = a.stream_tag;
+    p.codes = a.codes; p.scales = a.scales; p.sf_native = a.sf_native; p.y_out = a.y_out;
+    int dev = 0, sms = 0;
+    cudaError_t e = cudaGetDevice(&dev);
+    if (e != cudaSuccess) return e;
+    e = cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
+    if (e != cudaSuccess) return e;
+    const int64_t tiles = p.r_tiles * p.k_tiles;
+    const unsigned grid = (unsigned)(tiles < sms ? tiles : sms);
+    if (dump_y)
+        quantize_tc_kernel<true><<<grid, kThreadsQ, kSmemQ, stream>>>(a.tmap_x, p);
+    else
+        quantize_tc_kernel<false><<<grid, kThreadsQ, kSmemQ, stream>>>(a.tmap_x, p);
+    return cudaGetLastError();
+}
+
+}  // namespace mx
