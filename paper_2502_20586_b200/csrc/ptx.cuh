@@ -58,17 +58,30 @@ __device__ __forceinline__ uint64_t global_timer_ns() {
     asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t));
     return t;
 }
-__device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity, const volatile uint32_t* abort = nullptr) {
-    if (mbar_try_wait(bar, parity)) return true;
+// try_wait with a suspend-time hint: the hardware may park the thread for up to `hint_ns` while the phase is
+// pending, so a waiting role does not burn issue slots that the working warps of the CTA need.
+__device__ __forceinline__ bool mbar_try_wait_hint(uint64_t* bar, uint32_t parity, uint32_t hint_ns) {
+    uint32_t ok;
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2, %3;\n\t"
+        "selp.u32 %0, 1, 0, p;\n\t}"
+        : "=r"(ok) : "r"(smem_u32(bar)), "r"(parity), "r"(hint_ns) : "memory");
+    return ok != 0;
+}
+static __device__ __noinline__ bool mbar_wait_slow(uint64_t* bar, uint32_t parity, const volatile uint32_t* abort) {
     const uint64_t t0 = global_timer_ns();
     for (uint32_t i = 0;; ++i) {
-        if (mbar_try_wait(bar, parity)) return true;
+        if (mbar_try_wait_hint(bar, parity, 2000u)) return true;
         if (abort != nullptr && *abort != 0u) return false;
-        if (i > 32) __nanosleep(40);
-        if ((i & 63u) == 63u && global_timer_ns() - t0 > kWaitLimitNs) break;
+        if ((i & 15u) == 15u && global_timer_ns() - t0 > kWaitLimitNs) break;
     }
     atomicOr(&g_device_status, kStatusTimeout);
     return false;
+}
+__device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity, const volatile uint32_t* abort = nullptr) {
+    if (mbar_try_wait(bar, parity)) return true;
+    return mbar_wait_slow(bar, parity, abort);
 }
 
 // ---------------------------------------------------------------- TMA

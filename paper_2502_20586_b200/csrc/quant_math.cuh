@@ -133,8 +133,9 @@ __device__ __forceinline__ uint32_t pack8_from_half_sums(uint32_t s0, uint32_t s
 //     One 32-bit add handles two lanes (no carry can cross: the magnitude field is at most 0x0dff + 0x1ff).
 //   RN (Algorithm 1): hardware nearest-even convert of y / X.
 // A NaN input is out of contract (the block's scale is then taken from the other values); Inf gives byte 255.
-__device__ __forceinline__ void quantize_block32(const float (&y)[32], int rounding, uint64_t seed, uint32_t stream_tag,
-                                                 uint64_t i0, uint32_t (&packed)[4], uint32_t& scale_byte) {
+// `rw` holds the block's 32 SR draws (sr_draws32); it is not read when rounding = RN.
+__device__ __forceinline__ void quantize_block32_rw(const float (&y)[32], int rounding, const uint32_t (&rw)[8],
+                                                    uint32_t (&packed)[4], uint32_t& scale_byte) {
     float amax = 0.0f;
 #pragma unroll
     for (int i = 0; i < 32; i += 2) amax = fmaxf(amax, fmaxf(fabsf(y[i]), fabsf(y[i + 1])));
@@ -145,8 +146,6 @@ __device__ __forceinline__ void quantize_block32(const float (&y)[32], int round
     }
     const int e = (int)scale_byte - 127;
     if (rounding == 0) {
-        uint32_t rw[8];
-        sr_draws32(seed, stream_tag, i0, rw);
         if (e <= 100) {
             const float c = 1.5f * pow2f_wide(-e - 15);              // 3/4 * 2^(-e-14), a normal fp32
 #pragma unroll
@@ -188,6 +187,14 @@ __device__ __forceinline__ void quantize_block32(const float (&y)[32], int round
             packed[q] = word;
         }
     }
+}
+
+// Same, drawing the block's SR bits itself; i0 = linear index of the block's first element in the K-major operand.
+__device__ __forceinline__ void quantize_block32(const float (&y)[32], int rounding, uint64_t seed, uint32_t stream_tag,
+                                                 uint64_t i0, uint32_t (&packed)[4], uint32_t& scale_byte) {
+    uint32_t rw[8] = {0u, 0u, 0u, 0u, 0u, 0u, 0u, 0u};
+    if (rounding == 0) sr_draws32(seed, stream_tag, i0, rw);
+    quantize_block32_rw(y, rounding, rw, packed, scale_byte);
 }
 
 // Byte offset of the scale of (row r, 32-block k) in the tcgen05 scale-factor tiling: 128-row x 4-block

@@ -13,8 +13,8 @@
 //
 //   warp 0        TMA producer (two 64-column x 128-row boxes per tile, 128-byte swizzle, 4-stage ring)
 //   warp 1        MMA issuer (8 K=16 MMAs per tile into one of four 128-column TMEM accumulators)
-//   warps 2..17   epilogue: warp = (TMEM lane quadrant, MX block): tcgen05.ld 32 columns, release the
-//                 accumulator, then scale / SR / pack / store
+//   warps 2..17   epilogue, two groups of eight warps on alternate tiles: warp = (TMEM lane quadrant, 64 columns):
+//                 tcgen05.ld 32 columns at a time, release the accumulator, then scale / SR / pack / store
 // Every mbarrier wait is bounded; on expiry the CTA records a status word and unwinds.
 #include <cuda_bf16.h>
 
@@ -76,7 +76,7 @@ quantize_tc_kernel(const __grid_constant__ CUtensorMap tmap_x, const QParams p) 
 
     if (threadIdx.x == 0) {
         for (int s = 0; s < kStagesQ; ++s) { mbar_init(&full_bar[s], 1); mbar_init(&empty_bar[s], 1); }
-        for (int b = 0; b < kAccBufs; ++b) { mbar_init(&acc_full[b], 1); mbar_init(&acc_empty[b], kEpiWarps); }
+        for (int b = 0; b < kAccBufs; ++b) { mbar_init(&acc_full[b], 1); mbar_init(&acc_empty[b], kEpiWarps / 2); }
         *abort_flag = 0;
         mbar_fence_init();
         prefetch_tensormap(&tmap_x);
@@ -166,46 +166,101 @@ quantize_tc_kernel(const __grid_constant__ CUtensorMap tmap_x, const QParams p) 
         }
     } else {
         // ------------------------------------------------------------------ epilogue
+        // Two groups of eight warps take alternate tiles (so one group's integer-heavy packing overlaps the other's
+        // multiply-heavy Philox rounds); inside a group a warp owns one TMEM lane quadrant and 64 of the 128 columns,
+        // i.e. two MX blocks per thread and tile.  The SR draws of the NEXT tile are computed while the current one
+        // is rounded: they depend only on element indices.
         const int e = warp - 2;
         const int q = warp & 3;                      // TMEM lane quadrant this warp may read
-        const int blk = e >> 2;                      // MX block (32 columns) of the tile; q takes all four values within each blk
+        const int grp = e >> 3;
+        const int half = (e >> 2) & 1;
         const float cg = p.g == 32 ? 0.17677669529663687f : p.g == 128 ? 0.08838834764831845f : 1.0f;
-        const int64_t nkb = p.K >> 5, nkc = (nkb + 3) >> 2;
-        uint32_t it = 0;
+        const uint32_t k_tiles = (uint32_t)p.k_tiles, r_tiles = (uint32_t)p.r_tiles;
+        const uint32_t nkb = (uint32_t)(p.K >> 5), nkc = (nkb + 3) >> 2;
+        const bool sr = !DUMP_Y && p.rounding == 0;
+        const uint32_t ntile = (uint32_t)num_tiles, stride = 2u * gridDim.x;
+        const uint32_t lane_row = (uint32_t)(q * 32 + lane);
         bool ok = true;
-        for (int64_t t = blockIdx.x; t < num_tiles; t += gridDim.x, ++it) {
+
+        auto split = [&](uint32_t t, uint32_t& rt, uint32_t& kt) {
+            if (p.reduce_dim == 1) { rt = t / k_tiles; kt = t - rt * k_tiles; }
+            else { kt = t / r_tiles; rt = t - kt * r_tiles; }
+        };
+        auto first_elem = [&](uint32_t t) -> uint64_t {          // linear index of this thread's first element of tile t
+            uint32_t rt, kt;
+            split(t, rt, kt);
+            return (uint64_t)(rt * (uint32_t)kTile + lane_row) * (uint64_t)p.K + (uint64_t)(kt * (uint32_t)kTile + (uint32_t)half * 64u);
+        };
+
+        uint32_t it = (uint32_t)grp;
+        uint32_t t = blockIdx.x + it * gridDim.x;
+        uint32_t rw0[8], rw1[8];
+        if (sr && t < ntile) {
+            const uint64_t i0 = first_elem(t);
+            sr_draws32(p.seed, p.stream_tag, i0, rw0);
+            sr_draws32(p.seed, p.stream_tag, i0 + 32, rw1);
+        }
+        for (; t < ntile; t += stride, it += 2) {
             const int b = it % kAccBufs;
-            int64_t rt, kt;
-            if (p.reduce_dim == 1) { rt = t / p.k_tiles; kt = t - rt * p.k_tiles; }
-            else { kt = t / p.r_tiles; rt = t - kt * p.r_tiles; }
+            uint32_t rt, kt;
+            split(t, rt, kt);
+            const int64_t row = (int64_t)rt * kTile + lane_row;                 // output row
+            const int64_t k0 = (int64_t)kt * kTile + half * 64;
+            const bool live = row < p.R;
+            const bool more = sr && t + stride < ntile;
+            const uint64_t i_next = more ? first_elem(t + stride) : 0;
             ok = mbar_wait(&acc_full[b], (it / kAccBufs) & 1, abort_flag);
             ok = __all_sync(0xffffffffu, ok);
             if (!ok) break;
             tc_fence_after_sync();
-            uint32_t raw[32];
-            tmem_ld_32x32b_x32(tmem_base + ((uint32_t)(q * 32) << 16) + b * kTile + blk * 32, raw);
+            const uint32_t taddr = tmem_base + ((uint32_t)(q * 32) << 16) + b * kTile + half * 64;
+            uint32_t raw[32], n0[8], n1[8], packed[4], sb0 = 0, sb1 = 0;
+            float y[32];
+            // ---- first MX block
+            tmem_ld_32x32b_x32(taddr, raw);
+            tmem_ld_wait();
+            if (more) sr_draws32(p.seed, p.stream_tag, i_next, n0);
+#pragma unroll
+            for (int i = 0; i < 32; ++i) y[i] = __uint_as_float(raw[i]) * cg;   // exact no-op unless g is 32 or 128
+            if (DUMP_Y) {
+                if (live) {
+                    float4* dst = reinterpret_cast<float4*>(p.y_out + row * p.K + k0);
+#pragma unroll
+                    for (int i = 0; i < 8; ++i) dst[i] = make_float4(y[4 * i], y[4 * i + 1], y[4 * i + 2], y[4 * i + 3]);
+                }
+            } else {
+                quantize_block32_rw(y, p.rounding, rw0, packed, sb0);
+                if (live)
+                    *reinterpret_cast<uint4*>(p.codes + row * (p.K >> 1) + (k0 >> 1)) = make_uint4(packed[0], packed[1], packed[2], packed[3]);
+            }
+            // ---- second MX block; the accumulator is free once it has been read
+            tmem_ld_32x32b_x32(taddr + 32, raw);
             tmem_ld_wait();
             tc_fence_before_sync();
             __syncwarp();
             if (lane == 0) mbar_arrive(&acc_empty[b]);
-            const int64_t row = rt * kTile + q * 32 + lane;            // output row
-            if (row >= p.R) continue;
-            float y[32];
+            if (more) sr_draws32(p.seed, p.stream_tag, i_next + 32, n1);
 #pragma unroll
-            for (int i = 0; i < 32; ++i) y[i] = __uint_as_float(raw[i]) * cg;   // exact no-op unless g is 32 or 128
-            const int64_t k0 = kt * kTile + blk * 32;
+            for (int i = 0; i < 32; ++i) y[i] = __uint_as_float(raw[i]) * cg;
             if (DUMP_Y) {
-                float4* dst = reinterpret_cast<float4*>(p.y_out + row * p.K + k0);
+                if (live) {
+                    float4* dst = reinterpret_cast<float4*>(p.y_out + row * p.K + k0 + 32);
 #pragma unroll
-                for (int i = 0; i < 8; ++i) dst[i] = make_float4(y[4 * i], y[4 * i + 1], y[4 * i + 2], y[4 * i + 3]);
-                continue;
+                    for (int i = 0; i < 8; ++i) dst[i] = make_float4(y[4 * i], y[4 * i + 1], y[4 * i + 2], y[4 * i + 3]);
+                }
+            } else {
+                quantize_block32_rw(y, p.rounding, rw1, packed, sb1);
+                if (live) {
+                    *reinterpret_cast<uint4*>(p.codes + row * (p.K >> 1) + (k0 >> 1) + 16) = make_uint4(packed[0], packed[1], packed[2], packed[3]);
+                    const int64_t so = p.sf_native ? ((int64_t)(rt * nkc + kt) * 512 + lane * 16 + q * 4 + half * 2)
+                                                   : row * nkb + (k0 >> 5);
+                    *reinterpret_cast<uint16_t*>(p.scales + so) = (uint16_t)(sb0 | (sb1 << 8));
+                }
             }
-            uint32_t packed[4], sbyte;
-            quantize_block32(y, p.rounding, p.seed, p.stream_tag, (uint64_t)(row * p.K + k0), packed, sbyte);
-            *reinterpret_cast<uint4*>(p.codes + row * (p.K >> 1) + (k0 >> 1)) = make_uint4(packed[0], packed[1], packed[2], packed[3]);
-            const int64_t kb = k0 >> 5;
-            const int64_t so = p.sf_native ? ((rt * nkc + kt) * 512 + lane * 16 + q * 4 + blk) : row * nkb + kb;
-            p.scales[so] = (uint8_t)sbyte;
+            if (more) {
+#pragma unroll
+                for (int i = 0; i < 8; ++i) { rw0[i] = n0[i]; rw1[i] = n1[i]; }
+            }
         }
         if (!ok && lane == 0) *abort_flag = 1;
     }
@@ -226,7 +281,9 @@ quantize_tc_kernel(const __grid_constant__ CUtensorMap tmap_x, const QParams p) 
 
 bool quant_tc_eligible(const QuantArgs& a) {
     const int64_t K = a.reduce_dim == 1 ? a.cols : a.rows;
-    return (a.g == 32 || a.g == 64 || a.g == 128) && K % kTile == 0 && a.has_tmap;
+    const int64_t R = a.reduce_dim == 1 ? a.rows : a.cols;
+    const int64_t tiles = ((R + kTile - 1) / kTile) * (K / kTile);          // tile indices are 32-bit in the kernel
+    return (a.g == 32 || a.g == 64 || a.g == 128) && K % kTile == 0 && tiles < (int64_t(1) << 30) && a.has_tmap;
 }
 
 cudaError_t quant_tc_init() {
