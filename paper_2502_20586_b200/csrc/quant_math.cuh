@@ -43,6 +43,41 @@ __device__ __forceinline__ void sr_draws32(uint64_t seed, uint32_t stream_tag, u
     rw[4] = b.x; rw[5] = b.y; rw[6] = b.z; rw[7] = b.w;
 }
 
+// Same draws with the ten round keys expanded once per thread (they depend on the seed only).
+struct PhiloxKeys {
+    uint32_t k0[10], k1[10];
+};
+__device__ __forceinline__ PhiloxKeys philox_expand_keys(uint64_t seed) {
+    PhiloxKeys ks;
+    uint32_t a = (uint32_t)seed, b = (uint32_t)(seed >> 32);
+#pragma unroll
+    for (int i = 0; i < 10; ++i) {
+        ks.k0[i] = a; ks.k1[i] = b;
+        a += 0x9E3779B9u; b += 0xBB67AE85u;
+    }
+    return ks;
+}
+__device__ __forceinline__ uint4 philox4x32_10(uint32_t c0, uint32_t c1, uint32_t c2, uint32_t c3, const PhiloxKeys& ks) {
+#pragma unroll
+    for (int i = 0; i < 10; ++i) {
+        const uint32_t hi0 = __umulhi(0xD2511F53u, c0), lo0 = 0xD2511F53u * c0;
+        const uint32_t hi1 = __umulhi(0xCD9E8D57u, c2), lo1 = 0xCD9E8D57u * c2;
+        c0 = hi1 ^ c1 ^ ks.k0[i];
+        c1 = lo1;
+        c2 = hi0 ^ c3 ^ ks.k1[i];
+        c3 = lo0;
+    }
+    return make_uint4(c0, c1, c2, c3);
+}
+// i0 is a multiple of 32, so the two call indices i0/16 and i0/16 + 1 differ in the lowest bit only.
+__device__ __forceinline__ void sr_draws32(const PhiloxKeys& ks, uint32_t stream_tag, uint64_t i0, uint32_t (&rw)[8]) {
+    const uint32_t lo = (uint32_t)(i0 >> 4), hi = (uint32_t)(i0 >> 36);
+    const uint4 a = philox4x32_10(lo, hi, stream_tag, 1u, ks);
+    const uint4 b = philox4x32_10(lo | 1u, hi, stream_tag, 1u, ks);
+    rw[0] = a.x; rw[1] = a.y; rw[2] = a.z; rw[3] = a.w;
+    rw[4] = b.x; rw[5] = b.y; rw[6] = b.z; rw[7] = b.w;
+}
+
 // ---------------------------------------------------------------- Hadamard butterflies (Eq. 4)
 // In-place Sylvester transform over the 32 values of one thread (natural order, un-normalised).
 __device__ __forceinline__ void fwht32(float (&v)[32]) {
@@ -113,68 +148,91 @@ __device__ __forceinline__ uint32_t cvt_f16x2_rz(float lo, float hi) {
     return d;
 }
 
-// Eight SR-rounded values, held as four packed-half sums (bit 15 sign, bits 11:9 E2M1 magnitude code in each
-// 16-bit lane), to one 32-bit word of eight 4-bit codes, element 0 in the low nibble.
-__device__ __forceinline__ uint32_t pack8_from_half_sums(uint32_t s0, uint32_t s1, uint32_t s2, uint32_t s3) {
-    const uint32_t x = __byte_perm(s0, s1, 0x7531), y = __byte_perm(s2, s3, 0x7531);   // high byte of every lane: s000cccm
-    const uint32_t vx = (x >> 1) & 0x47474747u, vy = (y >> 1) & 0x47474747u;          // 0s000ccc
-    const uint32_t nx = (vx | (vx >> 3)) & 0x0F0F0F0Fu, ny = (vy | (vy >> 3)) & 0x0F0F0F0Fu;   // 0000sccc
-    const uint32_t ux = nx | (nx >> 4), uy = ny | (ny >> 4);                          // bytes 0 and 2: two nibbles each
-    return __byte_perm(ux, uy, 0x6420);
-}
+// Pipe balance: on this SM the integer/logic pipe issues a warp every other cycle while the FMA pipe (which also
+// executes IMAD) issues every cycle.  `k` carries two constants the compiler must not see (they arrive as kernel
+// parameters), so that the lane arithmetic below stays two multiply-adds instead of shift/add chains.
+struct PipeConsts {
+    uint32_t eight;    // 8
+    uint32_t neg16;    // 0xFFFFFFF0
+};
+__host__ __device__ inline PipeConsts make_pipe_consts() { return PipeConsts{8u, 0xFFFFFFF0u}; }
 
 // Quantise 32 consecutive fp32 values (one MX block) to 16 bytes of packed E2M1 codes + one E8M0 byte.
 //   SR (Algorithm 2): round up iff 256 frac >= r + 1/2 (Eq. 2 with an 8-bit dither), decided on the exact real
-//     w = (3/4) y / X.  Fast path: z = RZ(y * 3/4 * 2^(-e-14)) is truncated to fp16 (two values per cvt).  The
-//     factor 2^-14 places E2M1's subnormal/normal boundary on fp16's, so in each 16-bit lane bits 11:9 are the
-//     E2M1 code of the lower neighbour and the low 9 bits are floor(512 frac); adding 511 - 2r carries into bit 9
-//     exactly when floor(512 frac) >= 2r + 1, i.e. when 256 frac >= r + 1/2.  Both truncations are toward zero
-//     and every threshold is a multiple of the fp16 spacing, so the decision is that of the exact real.
-//     One 32-bit add handles two lanes (no carry can cross: the magnitude field is at most 0x0dff + 0x1ff).
+//     w = (3/4) y / X.  Fast path: z = RZ(y * 3/4 * 2^(-e-14)) is truncated to fp16, two values per cvt.  The
+//     factor 2^-14 places E2M1's subnormal/normal boundary on fp16's, so each 16-bit lane reads
+//         s 000 ccc fffffffff      ccc = E2M1 code of the lower neighbour, f = floor(512 frac).
+//     The lane is multiplied by 8 (0 ccc fffffffff 000; the sign falls into dead low bits of the next lane) and
+//     8 (511 - 2r) is added: the carry into ccc is set exactly when f >= 2r + 1, i.e. 256 frac >= r + 1/2.  Both
+//     truncations are toward zero and every threshold is a multiple of the fp16 spacing, so the decision is that
+//     of the exact real.  One 32-bit multiply-add handles two lanes; re-inserting the sign bits from the cvt
+//     result leaves the finished 4-bit code s ccc in the top nibble of each lane, so eight codes are gathered
+//     with two byte permutes, one shift and one select.  Lanes pair elements (i, i+2) and (i+1, i+3), which is
+//     how the four draws of one Philox word split with one mask and one byte permute.
 //   RN (Algorithm 1): hardware nearest-even convert of y / X.
+// `rw` holds the block's 32 SR draws (sr_draws32); it is not read when ROUNDING = 1 (RN).
 // A NaN input is out of contract (the block's scale is then taken from the other values); Inf gives byte 255.
-// `rw` holds the block's 32 SR draws (sr_draws32); it is not read when rounding = RN.
-__device__ __forceinline__ void quantize_block32_rw(const float (&y)[32], int rounding, const uint32_t (&rw)[8],
-                                                    uint32_t (&packed)[4], uint32_t& scale_byte) {
-    float amax = 0.0f;
-#pragma unroll
-    for (int i = 0; i < 32; i += 2) amax = fmaxf(amax, fmaxf(fabsf(y[i]), fabsf(y[i + 1])));
-    scale_byte = e8m0_from_amax(amax);
+__device__ __forceinline__ void quantize_block32_rare(const float (&y)[32], uint32_t scale_byte, const uint32_t (&rw)[8],
+                                                   uint32_t (&packed)[4]) {
+    // scale exponent above 100 (|values| beyond 2^103) or a non-finite block
     if (scale_byte == 255u) {
         packed[0] = packed[1] = packed[2] = packed[3] = 0u;
         return;
     }
     const int e = (int)scale_byte - 127;
-    if (rounding == 0) {
-        if (e <= 100) {
-            const float c = 1.5f * pow2f_wide(-e - 15);              // 3/4 * 2^(-e-14), a normal fp32
+    const int h1 = (-e) / 2, h2 = -e - h1;                           // exact 2^-e in two steps
+    const float p1 = pow2f_wide(h1), p2 = pow2f_wide(h2);
 #pragma unroll
-            for (int q = 0; q < 4; ++q) {
-                uint32_t s[4];
+    for (int q = 0; q < 4; ++q) {
+        uint32_t word = 0u;
 #pragma unroll
-                for (int p = 0; p < 4; ++p) {
-                    const int i = 8 * q + 2 * p;
-                    const uint32_t h = cvt_f16x2_rz(__fmul_rz(y[i], c), __fmul_rz(y[i + 1], c));
-                    const uint32_t x = __byte_perm(rw[i >> 2], 0u, (p & 1) ? 0x4342 : 0x4140);   // r_i | r_{i+1} << 16
-                    s[p] = h + (0x01FF01FFu - 2u * x);
-                }
-                packed[q] = pack8_from_half_sums(s[0], s[1], s[2], s[3]);
+        for (int j = 0; j < 8; ++j) {
+            const int i = 8 * q + j;
+            word |= sr_encode_wide(y[i], p1, p2, (rw[i >> 2] >> (8 * (i & 3))) & 0xFFu) << (4 * j);
+        }
+        packed[q] = word;
+    }
+}
+
+template <int ROUNDING>
+__device__ __forceinline__ void quantize_block32_rw(const float (&y)[32], const uint32_t (&rw)[8],
+                                                    uint32_t (&packed)[4], uint32_t& scale_byte, const PipeConsts& k) {
+    float amax = 0.0f;
+#pragma unroll
+    for (int i = 0; i < 32; i += 2) amax = fmaxf(amax, fmaxf(fabsf(y[i]), fabsf(y[i + 1])));
+    scale_byte = e8m0_from_amax(amax);
+    const int e = (int)scale_byte - 127;
+    if (ROUNDING == 0) {
+        if (scale_byte > 227u) {                                     // rare: keeps the common path branch-free
+            quantize_block32_rare(y, scale_byte, rw, packed);
+            return;
+        }
+        const float c = 1.5f * pow2f_wide(-e - 15);                  // 3/4 * 2^(-e-14), a normal fp32 since e <= 100
+#pragma unroll
+        for (int q = 0; q < 4; ++q) {
+            uint32_t u[4];
+#pragma unroll
+            for (int hh = 0; hh < 2; ++hh) {                         // four elements share one random word
+                const int i = 8 * q + 4 * hh;
+                const uint32_t w = rw[2 * q + hh];
+                const uint32_t r_even = w & 0x00FF00FFu;                     // r_i      | r_{i+2} << 16
+                const uint32_t r_odd = __byte_perm(w, 0u, 0x4341);           // r_{i+1}  | r_{i+3} << 16
+                const uint32_t h_even = cvt_f16x2_rz(__fmul_rz(y[i], c), __fmul_rz(y[i + 2], c));
+                const uint32_t h_odd = cvt_f16x2_rz(__fmul_rz(y[i + 1], c), __fmul_rz(y[i + 3], c));
+                const uint32_t t_even = h_even * k.eight + (r_even * k.neg16 + 0x0FF80FF8u);   // + 8 (511 - 2r) per lane
+                const uint32_t t_odd = h_odd * k.eight + (r_odd * k.neg16 + 0x0FF80FF8u);
+                u[hh] = (t_even & 0x7FFF7FFFu) | (h_even & 0x80008000u);     // s ccc .... in the top nibble of each lane
+                u[2 + hh] = (t_odd & 0x7FFF7FFFu) | (h_odd & 0x80008000u);
             }
-        } else {
-            const int h1 = (-e) / 2, h2 = -e - h1;                   // exact 2^-e in two steps
-            const float p1 = pow2f_wide(h1), p2 = pow2f_wide(h2);
-#pragma unroll
-            for (int q = 0; q < 4; ++q) {
-                uint32_t word = 0u;
-#pragma unroll
-                for (int j = 0; j < 8; ++j) {
-                    const int i = 8 * q + j;
-                    word |= sr_encode_wide(y[i], p1, p2, (rw[i >> 2] >> (8 * (i & 3))) & 0xFFu) << (4 * j);
-                }
-                packed[q] = word;
-            }
+            const uint32_t ev = __byte_perm(u[0], u[1], 0x7531);             // top bytes of elements 0, 2, 4, 6
+            const uint32_t od = __byte_perm(u[2], u[3], 0x7531);             // top bytes of elements 1, 3, 5, 7
+            packed[q] = ((ev >> 4) & 0x0F0F0F0Fu) | (od & 0xF0F0F0F0u);
         }
     } else {
+        if (scale_byte == 255u) {
+            packed[0] = packed[1] = packed[2] = packed[3] = 0u;
+            return;
+        }
         const float inv_x = pow2f_wide(-e);
 #pragma unroll
         for (int q = 0; q < 4; ++q) {
@@ -193,8 +251,12 @@ __device__ __forceinline__ void quantize_block32_rw(const float (&y)[32], int ro
 __device__ __forceinline__ void quantize_block32(const float (&y)[32], int rounding, uint64_t seed, uint32_t stream_tag,
                                                  uint64_t i0, uint32_t (&packed)[4], uint32_t& scale_byte) {
     uint32_t rw[8] = {0u, 0u, 0u, 0u, 0u, 0u, 0u, 0u};
-    if (rounding == 0) sr_draws32(seed, stream_tag, i0, rw);
-    quantize_block32_rw(y, rounding, rw, packed, scale_byte);
+    if (rounding == 0) {
+        sr_draws32(seed, stream_tag, i0, rw);
+        quantize_block32_rw<0>(y, rw, packed, scale_byte, make_pipe_consts());
+    } else {
+        quantize_block32_rw<1>(y, rw, packed, scale_byte, make_pipe_consts());
+    }
 }
 
 // Byte offset of the scale of (row r, 32-block k) in the tcgen05 scale-factor tiling: 128-row x 4-block

@@ -45,6 +45,8 @@ struct QParams {
     uint8_t* scales;
     int sf_native;
     float* y_out;
+    PipeConsts pipe;          // see quant_math.cuh: constants kept opaque to the compiler
+    PhiloxKeys keys;          // the ten Philox round keys of `seed` (key schedule only; the rounds run on the device)
 };
 
 // bf16 entry (n, k) of the transform operand, stored N x K (K-major): T[k][n] = S_k H_g[k][n] inside a g-chunk.
@@ -57,7 +59,9 @@ __device__ __forceinline__ uint32_t transform_entry(int n, int k, int g, const u
     return mag | (neg << 15);
 }
 
-template <bool DUMP_Y>
+enum { kModeSR = 0, kModeRN = 1, kModeDump = 2 };
+
+template <int MODE>
 __global__ void __launch_bounds__(kThreadsQ, 1)
 quantize_tc_kernel(const __grid_constant__ CUtensorMap tmap_x, const QParams p) {
     extern __shared__ uint8_t smem_raw[];
@@ -177,38 +181,39 @@ quantize_tc_kernel(const __grid_constant__ CUtensorMap tmap_x, const QParams p) 
         const float cg = p.g == 32 ? 0.17677669529663687f : p.g == 128 ? 0.08838834764831845f : 1.0f;
         const uint32_t k_tiles = (uint32_t)p.k_tiles, r_tiles = (uint32_t)p.r_tiles;
         const uint32_t nkb = (uint32_t)(p.K >> 5), nkc = (nkb + 3) >> 2;
-        const bool sr = !DUMP_Y && p.rounding == 0;
         const uint32_t ntile = (uint32_t)num_tiles, stride = 2u * gridDim.x;
         const uint32_t lane_row = (uint32_t)(q * 32 + lane);
         bool ok = true;
 
-        auto split = [&](uint32_t t, uint32_t& rt, uint32_t& kt) {
-            if (p.reduce_dim == 1) { rt = t / k_tiles; kt = t - rt * k_tiles; }
-            else { kt = t / r_tiles; rt = t - kt * r_tiles; }
-        };
-        auto first_elem = [&](uint32_t t) -> uint64_t {          // linear index of this thread's first element of tile t
-            uint32_t rt, kt;
-            split(t, rt, kt);
-            return (uint64_t)(rt * (uint32_t)kTile + lane_row) * (uint64_t)p.K + (uint64_t)(kt * (uint32_t)kTile + (uint32_t)half * 64u);
+        // Tile t -> (row tile, k tile) of the output operand; t advances by `stride` per iteration, so the
+        // coordinates are carried along instead of divided out each time.
+        const bool rowwise = p.reduce_dim == 1;
+        const uint32_t fast = rowwise ? k_tiles : r_tiles;                    // extent of the fast-running coordinate
+        const uint32_t dq = stride / fast, dr = stride - dq * fast;
+        const uint64_t K64 = (uint64_t)p.K;
+        auto first_elem = [&](uint32_t rt, uint32_t kt) -> uint64_t {        // linear index of this thread's first element
+            return (uint64_t)(rt * (uint32_t)kTile + lane_row) * K64 + (uint64_t)(kt * (uint32_t)kTile + (uint32_t)half * 64u);
         };
 
         uint32_t it = (uint32_t)grp;
         uint32_t t = blockIdx.x + it * gridDim.x;
+        uint32_t slow_c = t / fast, fast_c = t - slow_c * fast;               // one division per thread
         uint32_t rw0[8], rw1[8];
-        if (sr && t < ntile) {
-            const uint64_t i0 = first_elem(t);
-            sr_draws32(p.seed, p.stream_tag, i0, rw0);
-            sr_draws32(p.seed, p.stream_tag, i0 + 32, rw1);
+        if (MODE == kModeSR) {
+            const uint64_t i0 = rowwise ? first_elem(slow_c, fast_c) : first_elem(fast_c, slow_c);
+            sr_draws32(p.keys, p.stream_tag, i0, rw0);
+            sr_draws32(p.keys, p.stream_tag, i0 + 32, rw1);
         }
         for (; t < ntile; t += stride, it += 2) {
             const int b = it % kAccBufs;
-            uint32_t rt, kt;
-            split(t, rt, kt);
+            const uint32_t rt = rowwise ? slow_c : fast_c, kt = rowwise ? fast_c : slow_c;
+            fast_c += dr; slow_c += dq;
+            if (fast_c >= fast) { fast_c -= fast; ++slow_c; }                  // coordinates of tile t + stride
             const int64_t row = (int64_t)rt * kTile + lane_row;                 // output row
             const int64_t k0 = (int64_t)kt * kTile + half * 64;
             const bool live = row < p.R;
-            const bool more = sr && t + stride < ntile;
-            const uint64_t i_next = more ? first_elem(t + stride) : 0;
+            // draws of the next tile of this group (computed even past the end: they are simply not used)
+            const uint64_t i_next = rowwise ? first_elem(slow_c, fast_c) : first_elem(fast_c, slow_c);
             ok = mbar_wait(&acc_full[b], (it / kAccBufs) & 1, abort_flag);
             ok = __all_sync(0xffffffffu, ok);
             if (!ok) break;
@@ -216,22 +221,22 @@ quantize_tc_kernel(const __grid_constant__ CUtensorMap tmap_x, const QParams p) 
             const uint32_t taddr = tmem_base + ((uint32_t)(q * 32) << 16) + b * kTile + half * 64;
             uint32_t raw[32], n0[8], n1[8], packed[4], sb0 = 0, sb1 = 0;
             float y[32];
+            uint8_t* code_dst = p.codes + row * (p.K >> 1) + (k0 >> 1);
             // ---- first MX block
             tmem_ld_32x32b_x32(taddr, raw);
             tmem_ld_wait();
-            if (more) sr_draws32(p.seed, p.stream_tag, i_next, n0);
+            if (MODE == kModeSR) sr_draws32(p.keys, p.stream_tag, i_next, n0);
 #pragma unroll
             for (int i = 0; i < 32; ++i) y[i] = __uint_as_float(raw[i]) * cg;   // exact no-op unless g is 32 or 128
-            if (DUMP_Y) {
+            if (MODE == kModeDump) {
                 if (live) {
                     float4* dst = reinterpret_cast<float4*>(p.y_out + row * p.K + k0);
 #pragma unroll
                     for (int i = 0; i < 8; ++i) dst[i] = make_float4(y[4 * i], y[4 * i + 1], y[4 * i + 2], y[4 * i + 3]);
                 }
             } else {
-                quantize_block32_rw(y, p.rounding, rw0, packed, sb0);
-                if (live)
-                    *reinterpret_cast<uint4*>(p.codes + row * (p.K >> 1) + (k0 >> 1)) = make_uint4(packed[0], packed[1], packed[2], packed[3]);
+                quantize_block32_rw<MODE>(y, rw0, packed, sb0, p.pipe);
+                if (live) *reinterpret_cast<uint4*>(code_dst) = make_uint4(packed[0], packed[1], packed[2], packed[3]);
             }
             // ---- second MX block; the accumulator is free once it has been read
             tmem_ld_32x32b_x32(taddr + 32, raw);
@@ -239,25 +244,25 @@ quantize_tc_kernel(const __grid_constant__ CUtensorMap tmap_x, const QParams p) 
             tc_fence_before_sync();
             __syncwarp();
             if (lane == 0) mbar_arrive(&acc_empty[b]);
-            if (more) sr_draws32(p.seed, p.stream_tag, i_next + 32, n1);
+            if (MODE == kModeSR) sr_draws32(p.keys, p.stream_tag, i_next + 32, n1);
 #pragma unroll
             for (int i = 0; i < 32; ++i) y[i] = __uint_as_float(raw[i]) * cg;
-            if (DUMP_Y) {
+            if (MODE == kModeDump) {
                 if (live) {
                     float4* dst = reinterpret_cast<float4*>(p.y_out + row * p.K + k0 + 32);
 #pragma unroll
                     for (int i = 0; i < 8; ++i) dst[i] = make_float4(y[4 * i], y[4 * i + 1], y[4 * i + 2], y[4 * i + 3]);
                 }
             } else {
-                quantize_block32_rw(y, p.rounding, rw1, packed, sb1);
+                quantize_block32_rw<MODE>(y, rw1, packed, sb1, p.pipe);
                 if (live) {
-                    *reinterpret_cast<uint4*>(p.codes + row * (p.K >> 1) + (k0 >> 1) + 16) = make_uint4(packed[0], packed[1], packed[2], packed[3]);
+                    *reinterpret_cast<uint4*>(code_dst + 16) = make_uint4(packed[0], packed[1], packed[2], packed[3]);
                     const int64_t so = p.sf_native ? ((int64_t)(rt * nkc + kt) * 512 + lane * 16 + q * 4 + half * 2)
                                                    : row * nkb + (k0 >> 5);
                     *reinterpret_cast<uint16_t*>(p.scales + so) = (uint16_t)(sb0 | (sb1 << 8));
                 }
             }
-            if (more) {
+            if (MODE == kModeSR) {
 #pragma unroll
                 for (int i = 0; i < 8; ++i) { rw0[i] = n0[i]; rw1[i] = n1[i]; }
             }
@@ -287,9 +292,11 @@ bool quant_tc_eligible(const QuantArgs& a) {
 }
 
 cudaError_t quant_tc_init() {
-    cudaError_t e = cudaFuncSetAttribute(quantize_tc_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kSmemQ);
+    cudaError_t e = cudaFuncSetAttribute(quantize_tc_kernel<kModeSR>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kSmemQ);
     if (e != cudaSuccess) return e;
-    return cudaFuncSetAttribute(quantize_tc_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kSmemQ);
+    e = cudaFuncSetAttribute(quantize_tc_kernel<kModeRN>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kSmemQ);
+    if (e != cudaSuccess) return e;
+    return cudaFuncSetAttribute(quantize_tc_kernel<kModeDump>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kSmemQ);
 }
 
 cudaError_t launch_quantize_tc(const QuantArgs& a, bool dump_y, cudaStream_t stream) {
@@ -301,6 +308,14 @@ cudaError_t launch_quantize_tc(const QuantArgs& a, bool dump_y, cudaStream_t str
     p.reduce_dim = a.reduce_dim; p.g = a.g; p.rounding = a.rounding;
     p.seed = a.seed; p.stream_tag = a.stream_tag;
     p.codes = a.codes; p.scales = a.scales; p.sf_native = a.sf_native; p.y_out = a.y_out;
+    p.pipe = make_pipe_consts();
+    {   // Philox key schedule: key_i = key_0 + i * (0x9E3779B9, 0xBB67AE85)
+        uint32_t k0 = (uint32_t)a.seed, k1 = (uint32_t)(a.seed >> 32);
+        for (int i = 0; i < 10; ++i) {
+            p.keys.k0[i] = k0; p.keys.k1[i] = k1;
+            k0 += 0x9E3779B9u; k1 += 0xBB67AE85u;
+        }
+    }
     int dev = 0, sms = 0;
     cudaError_t e = cudaGetDevice(&dev);
     if (e != cudaSuccess) return e;
@@ -309,9 +324,11 @@ cudaError_t launch_quantize_tc(const QuantArgs& a, bool dump_y, cudaStream_t str
     const int64_t tiles = p.r_tiles * p.k_tiles;
     const unsigned grid = (unsigned)(tiles < sms ? tiles : sms);
     if (dump_y)
-        quantize_tc_kernel<true><<<grid, kThreadsQ, kSmemQ, stream>>>(a.tmap_x, p);
+        quantize_tc_kernel<kModeDump><<<grid, kThreadsQ, kSmemQ, stream>>>(a.tmap_x, p);
+    else if (a.rounding == 0)
+        quantize_tc_kernel<kModeSR><<<grid, kThreadsQ, kSmemQ, stream>>>(a.tmap_x, p);
     else
-        quantize_tc_kernel<false><<<grid, kThreadsQ, kSmemQ, stream>>>(a.tmap_x, p);
+        quantize_tc_kernel<kModeRN><<<grid, kThreadsQ, kSmemQ, stream>>>(a.tmap_x, p);
     return cudaGetLastError();
 }
 
