@@ -148,6 +148,13 @@ __device__ __forceinline__ uint32_t cvt_f16x2_rz(float lo, float hi) {
     return d;
 }
 
+// (a & ~mask) | (b & mask) in one LOP3.
+__device__ __forceinline__ uint32_t bitselect(uint32_t a, uint32_t b, uint32_t mask) {
+    uint32_t d;
+    asm("lop3.b32 %0, %1, %2, %3, 0xD8;" : "=r"(d) : "r"(a), "r"(b), "r"(mask));
+    return d;
+}
+
 // Pipe balance: on this SM the integer/logic pipe issues a warp every other cycle while the FMA pipe (which also
 // executes IMAD) issues every cycle.  `k` carries two constants the compiler must not see (they arrive as kernel
 // parameters), so that the lane arithmetic below stays two multiply-adds instead of shift/add chains.
@@ -221,12 +228,12 @@ __device__ __forceinline__ void quantize_block32_rw(const float (&y)[32], const 
                 const uint32_t h_odd = cvt_f16x2_rz(__fmul_rz(y[i + 1], c), __fmul_rz(y[i + 3], c));
                 const uint32_t t_even = h_even * k.eight + (r_even * k.neg16 + 0x0FF80FF8u);   // + 8 (511 - 2r) per lane
                 const uint32_t t_odd = h_odd * k.eight + (r_odd * k.neg16 + 0x0FF80FF8u);
-                u[hh] = (t_even & 0x7FFF7FFFu) | (h_even & 0x80008000u);     // s ccc .... in the top nibble of each lane
-                u[2 + hh] = (t_odd & 0x7FFF7FFFu) | (h_odd & 0x80008000u);
+                u[hh] = bitselect(t_even, h_even, 0x80008000u);              // s ccc .... in the top nibble of each lane
+                u[2 + hh] = bitselect(t_odd, h_odd, 0x80008000u);
             }
             const uint32_t ev = __byte_perm(u[0], u[1], 0x7531);             // top bytes of elements 0, 2, 4, 6
             const uint32_t od = __byte_perm(u[2], u[3], 0x7531);             // top bytes of elements 1, 3, 5, 7
-            packed[q] = ((ev >> 4) & 0x0F0F0F0Fu) | (od & 0xF0F0F0F0u);
+            packed[q] = bitselect(ev >> 4, od, 0xF0F0F0F0u);
         }
     } else {
         if (scale_byte == 255u) {
