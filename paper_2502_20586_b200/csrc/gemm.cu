@@ -6,8 +6,12 @@
 //   warp 0      TMA producer: per stage 128 B (256 elements) of K for 128 rows of A and 256 rows of B through
 //               128-byte-swizzled tensor maps, plus the scale tiles (already in the tcgen05 tiling in global
 //               memory) as plain bulk copies;
-//   warp 1      MMA issuer: scale tiles shared memory -> TMEM (tcgen05.cp), then four K = 64 MMAs per stage;
-//   warps 2..5  epilogue: TMEM -> registers (tcgen05.ld) -> alpha -> bf16/fp32 -> global.
+//   warp 1      MMA issuer: four K = 64 MMAs per stage;
+//   warps 2..5  epilogue: TMEM -> registers (tcgen05.ld) -> alpha -> bf16/fp32 -> global;
+//   warps 6..9  scale-factor movers: per stage, shared memory -> registers -> TMEM (tcgen05.st), one warp per
+//               TMEM lane quadrant (the MMA wants the scales replicated in all four).  Doing this with
+//               tcgen05.cp from the MMA thread put ~64 cycles per copy in series with the MMAs (six per step:
+//               measured 3.6 vs 5.25 PFLOP/s without them); tcgen05.st runs beside the MMA pipe.
 // Every mbarrier wait is bounded; on expiry the CTA records a status word and unwinds.
 #include <cuda_bf16.h>
 
@@ -24,16 +28,18 @@ constexpr int BM = kGemmBM, BN = kGemmBN;
 constexpr int kStages = 4;
 constexpr uint32_t kABytes = BM * kGemmBKBytes;             // 16 KB
 constexpr uint32_t kBBytes = BN * kGemmBKBytes;             // 32 KB
-constexpr uint32_t kSfChunk = 512;                          // 128 rows x 4 K-blocks
-constexpr uint32_t kSfaBytes = 2 * kSfChunk;                // 2 chunks per stage (8 K-blocks)
+constexpr uint32_t kSfChunk = 512;                          // scale tile: 128 rows x 4 K-blocks
+constexpr uint32_t kSfaBytes = 2 * kSfChunk;                // 2 tiles per stage (8 K-blocks)
 constexpr uint32_t kSfbBytes = (BN / 128) * 2 * kSfChunk;
 constexpr uint32_t kStageBytes = kABytes + kBBytes + kSfaBytes + kSfbBytes;   // 51 KB, multiple of 1024
 constexpr uint32_t kSmemBytes = kStages * kStageBytes + 1024 /*alignment slack*/ + 256 /*barriers*/;
 constexpr uint32_t kTmemCols = 512;
 constexpr uint32_t kAccCol = 0;                             // 256 fp32 accumulator columns
-constexpr uint32_t kSfCol = 256;                            // two slots of (8 SFA + 16 SFB) columns
+constexpr uint32_t kSfCol = 256;                            // kSfSlots slots of (8 SFA + 16 SFB) columns
 constexpr uint32_t kSfSlotCols = 24;
+constexpr int kSfSlots = 4;
 constexpr int kGroupM = 16;                                 // tile rasterisation: 16 m-tiles share B tiles in L2
+constexpr int kThreads = 10 * 32;
 
 struct Params {
     const uint8_t* sfa;
@@ -55,25 +61,30 @@ __device__ __forceinline__ void tile_coords(int t, int m_tiles, int n_tiles, int
     nt = r / gm;
 }
 
-__global__ void __launch_bounds__(192, 1)
+__global__ void __launch_bounds__(kThreads, 1)
 gemm_mxf4_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant__ CUtensorMap tmap_b, const Params p) {
     extern __shared__ uint8_t smem_raw[];
     uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
     uint64_t* bars = reinterpret_cast<uint64_t*>(smem + kStages * kStageBytes);
-    uint64_t* full_bar = bars;                    // [kStages] TMA -> MMA
-    uint64_t* empty_bar = bars + kStages;         // [kStages] MMA -> TMA
-    uint64_t* tmem_full = bars + 2 * kStages;     // MMA -> epilogue
-    uint64_t* tmem_empty = bars + 2 * kStages + 1;  // epilogue -> MMA
-    uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 2 * kStages + 2);
+    uint64_t* full_bar = bars;                              // [kStages]  TMA -> MMA, scale movers
+    uint64_t* empty_bar = full_bar + kStages;               // [kStages]  MMA -> TMA
+    uint64_t* sf_full = empty_bar + kStages;                // [kSfSlots] scale movers -> MMA
+    uint64_t* sf_empty = sf_full + kSfSlots;                // [kSfSlots] MMA -> scale movers
+    uint64_t* tmem_full = sf_empty + kSfSlots;              // MMA -> epilogue
+    uint64_t* tmem_empty = tmem_full + 1;                   // epilogue -> MMA
+    uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(tmem_empty + 1);
     volatile uint32_t* abort_flag = tmem_slot + 1;
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int num_tiles = p.m_tiles * p.n_tiles;
     const int nkc = (int)(p.K >> 7);                          // 128-element scale chunks along K
     const int num_kt = (nkc + 1) >> 1;                        // 256-element pipeline steps
+    const uint32_t my_tiles = blockIdx.x < (uint32_t)num_tiles ? ((uint32_t)num_tiles - blockIdx.x + gridDim.x - 1) / gridDim.x : 0u;
+    const uint32_t total = my_tiles * (uint32_t)num_kt;       // K-steps this CTA runs, over all its tiles
 
     if (threadIdx.x == 0) {
         for (int s = 0; s < kStages; ++s) { mbar_init(&full_bar[s], 1); mbar_init(&empty_bar[s], 1); }
+        for (int s = 0; s < kSfSlots; ++s) { mbar_init(&sf_full[s], 4); mbar_init(&sf_empty[s], 1); }
         mbar_init(tmem_full, 1);
         mbar_init(tmem_empty, 4);
         *abort_flag = 0;
@@ -121,41 +132,62 @@ gemm_mxf4_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_consta
         if (lane == 0) {
             // instruction descriptor: A, B = E2M1 (1), scale = UE8M0 (1), K-major, N >> 3 at bit 17, M >> 4 at bit 24
             const uint32_t idesc_base = (1u << 7) | (1u << 10) | ((uint32_t)(BN >> 3) << 17) | (1u << 23) | ((uint32_t)(BM >> 4) << 24);
-            uint32_t it = 0, tile_i = 0;
+            uint32_t tile_i = 0;
             bool ok = true;
-            for (int t = blockIdx.x; t < num_tiles && ok; t += gridDim.x, ++tile_i) {
-                if (!(ok = mbar_wait(tmem_empty, (tile_i & 1) ^ 1, abort_flag))) break;
-                tc_fence_after_sync();
-                for (int kt = 0; kt < num_kt; ++kt, ++it) {
-                    const int s = it % kStages;
-                    const uint32_t ph = (it / kStages) & 1;
-                    if (!(ok = mbar_wait(&full_bar[s], ph, abort_flag))) break;
-                    tc_fence_after_sync();
-                    const uint32_t st = smem_u32(smem + s * kStageBytes);
-                    const int nch = min(2, nkc - 2 * kt);
-                    const uint32_t sfa_t = tmem_base + kSfCol + (it & 1) * kSfSlotCols;
-                    const uint32_t sfb_t = sfa_t + 8;
-                    for (int c = 0; c < nch; ++c) {
-                        tc_cp_32x128b_warpx4(sfa_t + 4 * c, make_smem_desc(st + kABytes + kBBytes + c * kSfChunk, 0, 128, 0));
-                        for (int j = 0; j < BN / 128; ++j)
-                            tc_cp_32x128b_warpx4(sfb_t + 8 * c + 4 * j,
-                                                 make_smem_desc(st + kABytes + kBBytes + kSfaBytes + (j * 2 + c) * kSfChunk, 0, 128, 0));
-                    }
-                    for (int kb = 0; kb < 2 * nch; ++kb) {
-                        const uint64_t adesc = make_smem_desc(st + kb * 32, 16, 1024, 2);
-                        const uint64_t bdesc = make_smem_desc(st + kABytes + kb * 32, 16, 1024, 2);
-                        const uint32_t sf_id = (uint32_t)(kb & 1) * 2u;       // byte pair inside the 32-bit scale column
-                        const uint32_t idesc = idesc_base | (sf_id << 29) | (sf_id << 4);
-                        tc_mma_mxf4(tmem_base + kAccCol, adesc, bdesc, idesc,
-                                    (sfa_t + 4 * (kb >> 1)) | (sf_id << 30), (sfb_t + 8 * (kb >> 1)) | (sf_id << 30),
-                                    (kt | kb) != 0 ? 1u : 0u);
-                    }
-                    tc_commit(&empty_bar[s]);
+            for (uint32_t it = 0; it < total; ++it) {
+                const int kt = (int)(it % (uint32_t)num_kt);
+                const int s = it % kStages, slot = it % kSfSlots;
+                if (kt == 0) {
+                    if (!(ok = mbar_wait(tmem_empty, (tile_i & 1) ^ 1, abort_flag))) break;
                 }
-                if (ok) tc_commit(tmem_full);
+                if (!(ok = mbar_wait(&full_bar[s], (it / kStages) & 1, abort_flag))) break;
+                if (!(ok = mbar_wait(&sf_full[slot], (it / kSfSlots) & 1, abort_flag))) break;
+                tc_fence_after_sync();
+                const uint32_t st = smem_u32(smem + s * kStageBytes);
+                const int nch = min(2, nkc - 2 * kt);
+                const uint32_t sfa_t = tmem_base + kSfCol + slot * kSfSlotCols, sfb_t = sfa_t + 8;
+                for (int kb = 0; kb < 2 * nch; ++kb) {
+                    const uint64_t adesc = make_smem_desc(st + kb * 32, 16, 1024, 2);
+                    const uint64_t bdesc = make_smem_desc(st + kABytes + kb * 32, 16, 1024, 2);
+                    const uint32_t sf_id = (uint32_t)(kb & 1) * 2u;           // byte pair inside the 32-bit scale column
+                    const uint32_t idesc = idesc_base | (sf_id << 29) | (sf_id << 4);
+                    tc_mma_mxf4(tmem_base + kAccCol, adesc, bdesc, idesc,
+                                (sfa_t + 4 * (kb >> 1)) | (sf_id << 30), (sfb_t + 8 * (kb >> 1)) | (sf_id << 30),
+                                (kt | kb) != 0 ? 1u : 0u);
+                }
+                tc_commit(&empty_bar[s]);                                     // stage and scale slot are free once
+                tc_commit(&sf_empty[slot]);                                   // these MMAs have read them
+                if (kt == num_kt - 1) { tc_commit(tmem_full); ++tile_i; }
             }
             if (!ok) *abort_flag = 1;
         }
+    } else if (warp >= 6) {
+        // ------------------------------------------------------------------ scale-factor movers (warps 6..9)
+        // A 512-byte scale tile is the image of 32 TMEM lanes x 4 columns: lane l holds the 16 bytes at l * 16
+        // (rows l, l+32, l+64, l+96 of the 128-row tile, four K-blocks each).  Each warp writes that image into
+        // its own lane quadrant, which gives the four-fold replication the MMA expects.  Tiles the stage does
+        // not hold (K tail, N tail) leave stale bytes in columns whose products are never stored.
+        const int q = warp & 3;
+        const uint32_t lane_base = (uint32_t)(q * 32) << 16;
+        bool ok = true;
+        for (uint32_t it = 0; it < total; ++it) {
+            const int s = it % kStages, slot = it % kSfSlots;
+            ok = mbar_wait(&sf_empty[slot], ((it / kSfSlots) & 1) ^ 1, abort_flag) &&
+                 mbar_wait(&full_bar[s], (it / kStages) & 1, abort_flag);
+            ok = __all_sync(0xffffffffu, ok);
+            if (!ok) break;
+            tc_fence_after_sync();
+            const uint4* sf = reinterpret_cast<const uint4*>(smem + s * kStageBytes + kABytes + kBBytes) + lane;   // 32 uint4 per tile
+            const uint32_t sfa_t = tmem_base + lane_base + kSfCol + slot * kSfSlotCols, sfb_t = sfa_t + 8;
+            // stage layout: SFA tile 0, 1 | SFB (rows 0-127) tile 0, 1 | SFB (rows 128-255) tile 0, 1
+            tmem_st_32x32b_x8(sfa_t, sf[0], sf[32]);
+            tmem_st_32x32b_x16(sfb_t, sf[64], sf[128], sf[96], sf[160]);      // columns: (tile 0: rows 0-127 | 128-255) | (tile 1: ...)
+            tmem_st_wait();
+            tc_fence_before_sync();
+            __syncwarp();
+            if (lane == 0) mbar_arrive(&sf_full[slot]);
+        }
+        if (!ok && lane == 0) *abort_flag = 1;
     } else {
         // ------------------------------------------------------------------ epilogue (warps 2..5)
         const int q = warp & 3;                                   // TMEM lane quadrant this warp may read
@@ -243,7 +275,7 @@ cudaError_t launch_gemm(const GemmArgs& a, cudaStream_t stream) {
     if (e != cudaSuccess) return e;
     const int tiles = p.m_tiles * p.n_tiles;
     const int grid = tiles < sms ? tiles : sms;
-    gemm_mxf4_kernel<<<grid, 192, kSmemBytes, stream>>>(a.tmap_a, a.tmap_b, p);
+    gemm_mxf4_kernel<<<grid, kThreads, kSmemBytes, stream>>>(a.tmap_a, a.tmap_b, p);
     return cudaGetLastError();
 }
 
