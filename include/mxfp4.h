@@ -122,6 +122,31 @@ MXFP4_API mxfp4_status mxfp4_linear_backward(const void* dY, const void* X, cons
                                    void* dX, void* dW, int out_dtype,
                                    void* workspace, size_t workspace_bytes, void* cuda_stream);
 
+/*
+ * The same backward pass for callers that cannot supply a workspace.  (The paper has no counterpart: this is a
+ * property of the library, not of the method.)
+ *
+ * Who needs it: code that runs where device memory cannot be requested, for instance a hook called while its host
+ * framework's memory pool is locked or fully handed out, a plug-in that must not touch the CUDA allocator of the
+ * process it lives in, or a tool that has to keep working once device memory is exhausted.  Instead of a caller's
+ * buffer the scratch is a fixed array of MXFP4_STATIC_WORKSPACE_BYTES inside the library image; every GPU that loads
+ * the library holds that much memory from load to exit, whether or not this call is ever used.
+ *
+ *   Arguments and results are those of mxfp4_linear_backward without the workspace pair.
+ *   Shapes whose mxfp4_linear_backward_workspace(b, m, n) exceeds MXFP4_STATIC_WORKSPACE_BYTES are refused with
+ *   MXFP4_ERR_WORKSPACE; nothing is enqueued.
+ *   The call allocates nothing, neither on the host nor on the device.
+ *   The first call on each device looks up the array's device address (cudaGetSymbolAddress, with that device
+ *   current); make that first call outside any stream capture.
+ *   All calls on a device share the one array, which keeps whatever the previous call left in it.  Each call rewrites
+ *   every byte it later reads, so nothing needs clearing between calls; but two calls whose kernels can overlap on
+ *   the GPU (different streams without ordering) race on it: order them.
+ */
+#define MXFP4_STATIC_WORKSPACE_BYTES (8u << 20)
+MXFP4_API mxfp4_status mxfp4_linear_backward_static(const void* dY, const void* X, const void* W,
+                                                    int64_t b, int64_t m, int64_t n, int g, int rounding, uint64_t seed,
+                                                    void* dX, void* dW, int out_dtype, void* cuda_stream);
+
 /* Size in bytes of a scale tensor for an operand [rows, K] in the given layout (NATIVE is padded). */
 MXFP4_API size_t mxfp4_scale_bytes(int64_t rows, int64_t K, int sf_layout);
 

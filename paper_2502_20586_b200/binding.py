@@ -31,6 +31,8 @@ _lib.mxfp4_linear_backward_workspace.argtypes = [_i64, _i64, _i64]
 _lib.mxfp4_linear_backward_workspace.restype = _sz
 _lib.mxfp4_linear_backward.argtypes = [_vp, _vp, _vp, _i64, _i64, _i64, _int, _int, _u64, _vp, _vp, _int, _vp, _sz, _vp]
 _lib.mxfp4_linear_backward.restype = _int
+_lib.mxfp4_linear_backward_static.argtypes = [_vp, _vp, _vp, _i64, _i64, _i64, _int, _int, _u64, _vp, _vp, _int, _vp]
+_lib.mxfp4_linear_backward_static.restype = _int
 _lib.mxfp4_scale_bytes.argtypes = [_i64, _i64, _int]
 _lib.mxfp4_scale_bytes.restype = _sz
 _lib.mxfp4_device_status.argtypes = [_vp]
@@ -39,7 +41,7 @@ _lib.mxfp4_status_string.argtypes = [_int]
 _lib.mxfp4_status_string.restype = C.c_char_p
 
 EXPORTS = ["mxfp4_rht_sr_quantize", "mxfp4_rht", "mxfp4_gemm", "mxfp4_linear_backward_workspace",
-           "mxfp4_linear_backward", "mxfp4_scale_bytes", "mxfp4_device_status", "mxfp4_status_string"]
+           "mxfp4_linear_backward", "mxfp4_linear_backward_static", "mxfp4_scale_bytes", "mxfp4_device_status", "mxfp4_status_string"]
 
 
 class MxFp4Error(RuntimeError):
@@ -129,6 +131,28 @@ def mxfp4_linear_backward(dY, X, W, g: int, seed: int, rounding: int = ROUND_SR,
         workspace = torch.empty(need, dtype=torch.uint8, device=dY.device)
     _check(_lib.mxfp4_linear_backward(_ptr(dY), _ptr(X), _ptr(W), b, m, n, g, rounding, seed, _ptr(dX), _ptr(dW),
                                       out_dtype, _ptr(workspace), workspace.numel(), _stream()))
+    return dX, dW
+
+
+STATIC_WORKSPACE_BYTES = 8 << 20
+
+
+def mxfp4_linear_backward_static(dY, X, W, g: int, seed: int, rounding: int = ROUND_SR, out_dtype: int = OUT_BF16,
+                                 dX=None, dW=None):
+    """mxfp4_linear_backward for callers that cannot provide scratch memory: the library's own fixed array
+    (STATIC_WORKSPACE_BYTES per GPU) holds the quantised operands.  Pass dX and dW to make the call itself
+    allocation-free; shapes that need more scratch than the array raise MxFp4Error(6)."""
+    b, m = dY.shape
+    _, n = X.shape
+    for t in (dY, X, W):
+        assert t.is_cuda and t.dtype == torch.bfloat16 and t.is_contiguous()
+    dt = torch.float32 if out_dtype == OUT_FP32 else torch.bfloat16
+    if dX is None:
+        dX = torch.empty((b, n), dtype=dt, device=dY.device)
+    if dW is None:
+        dW = torch.empty((m, n), dtype=dt, device=dY.device)
+    _check(_lib.mxfp4_linear_backward_static(_ptr(dY), _ptr(X), _ptr(W), b, m, n, g, rounding, seed, _ptr(dX), _ptr(dW),
+                                             out_dtype, _stream()))
     return dX, dW
 
 
