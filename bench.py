@@ -150,6 +150,28 @@ def run_reference(args):
     }))
 
 
+# ------------------------------------------------------------------------------------------ multi-rank glue
+def rank_seed(seed: int, rank: int) -> int:
+    """Each rank draws its own tokens (data parallel): its input seed."""
+    return seed + rank
+
+
+def max_over_ranks(ms, ms_e2e, world: int, device):
+    """Step times of the whole job = the slowest rank's (no collective runs inside the timed path itself)."""
+    if world == 1:
+        return ms, ms_e2e
+    import torch
+    import torch.distributed as dist
+    t = torch.tensor([ms, ms_e2e or 0.0], device=device, dtype=torch.float64)
+    dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    return float(t[0]), (float(t[1]) if ms_e2e else None)
+
+
+def aggregate_value(flops_per_rank: float, world: int, ms: float) -> float:
+    """Whole-job TFLOP/s: every rank's FLOPs over the slowest rank's step time (weak scaling)."""
+    return world * flops_per_rank / (ms * 1e-3) / 1e12
+
+
 # ------------------------------------------------------------------------------------------------ GPU arm
 def run_gpu(args):
     import torch
@@ -176,7 +198,7 @@ def run_gpu(args):
     out_dtype = mx.OUT_BF16
     data = []
     for layer in layers:
-        dY, X, W = wl.layer_inputs_device(args.config, layer, seed=seed + rank, device=dev)
+        dY, X, W = wl.layer_inputs_device(args.config, layer, seed=rank_seed(seed, rank), device=dev)
         dX = torch.empty((layer.b, layer.n), dtype=torch.bfloat16, device=dev)
         dW = torch.empty((layer.m, layer.n), dtype=torch.bfloat16, device=dev)
         data.append((layer, dY, X, W, dX, dW))
@@ -301,12 +323,9 @@ def run_gpu(args):
         ms_e2e = e0.elapsed_time(e1) / k_e2e
 
     # ---- max over ranks
-    if world > 1:
-        t = torch.tensor([ms, ms_e2e or 0.0], device=dev, dtype=torch.float64)
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        ms, ms_e2e = float(t[0]), (float(t[1]) if ms_e2e else None)
-    value = world * flops_step / (ms * 1e-3) / 1e12
-    e2e_value = world * flops_step / (ms_e2e * 1e-3) / 1e12 if ms_e2e else None
+    ms, ms_e2e = max_over_ranks(ms, ms_e2e, world, dev)
+    value = aggregate_value(flops_step, world, ms)
+    e2e_value = aggregate_value(flops_step, world, ms_e2e) if ms_e2e else None
 
     cpu_baseline = None
     if rank == 0 and world == 1 and not args.no_cpu_baseline and "e2e" in legs:
