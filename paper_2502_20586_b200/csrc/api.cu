@@ -3,6 +3,7 @@
 #include <cuda_runtime.h>
 #include <stdint.h>
 
+#include <cstdlib>
 #include <mutex>
 
 #include "../../include/mxfp4.h"
@@ -22,6 +23,7 @@ struct Runtime {
     std::once_flag once;
     mxfp4_status status = MXFP4_OK;
     EncodeTiledFn encode = nullptr;
+    bool gemm_pair = true;       // CTA-pair GEMM unless MXFP4_GEMM_1CTA=1 (debugging / comparison)
 };
 Runtime g_rt;
 
@@ -45,7 +47,9 @@ mxfp4_status runtime_init() {
             return;
         }
         g_rt.encode = reinterpret_cast<EncodeTiledFn>(fn);
-        if (mx::gemm_init() != cudaSuccess || mx::quant_tc_init() != cudaSuccess) g_rt.status = MXFP4_ERR_CUDA;
+        if (mx::gemm_init() != cudaSuccess || mx::gemm_pair_init() != cudaSuccess || mx::quant_tc_init() != cudaSuccess) g_rt.status = MXFP4_ERR_CUDA;
+        const char* one_cta = getenv("MXFP4_GEMM_1CTA");
+        g_rt.gemm_pair = !(one_cta != nullptr && one_cta[0] == '1');
     });
     return g_rt.status;
 }
@@ -112,6 +116,12 @@ mxfp4_status gemm_impl(const uint8_t* A_codes, const uint8_t* A_scales, const ui
     a.sfa = A_scales; a.sfb = B_scales;
     a.M = M; a.N = N; a.K = K;
     a.alpha = alpha; a.C = C; a.ldc = ldc; a.out_fp32 = out_dtype == MXFP4_OUT_FP32;
+    a.use_pair = g_rt.gemm_pair && M > 128;                   // one 128-row tile gives a pair nothing to share
+    if (a.use_pair) {
+        st = make_codes_map(&a.tmap_b_half, B_codes, N, K, 128);
+        if (st != MXFP4_OK) return st;
+        return mx::launch_gemm_pair(a, stream) == cudaSuccess ? MXFP4_OK : MXFP4_ERR_CUDA;
+    }
     return mx::launch_gemm(a, stream) == cudaSuccess ? MXFP4_OK : MXFP4_ERR_CUDA;
 }
 

@@ -33,6 +33,8 @@ cudaError_t launch_rht_dump(const QuantArgs& a, cudaStream_t stream);
 struct GemmArgs {
     CUtensorMap tmap_a;   // codes [M, K/2] bytes, box 128 B x 128 rows, 128-byte swizzle
     CUtensorMap tmap_b;   // codes [N, K/2] bytes, box 128 B x BN rows
+    CUtensorMap tmap_b_half;   // same tensor, box 128 B x 128 rows (CTA-pair kernel: each CTA loads half a B tile)
+    bool use_pair;        // run the CTA-pair kernel (gemm_pair.cu)
     const uint8_t* sfa;   // native scale layout
     const uint8_t* sfb;
     int64_t M, N, K;
@@ -48,5 +50,7 @@ constexpr int kGemmBKBytes = 128;   // 256 E2M1 elements per pipeline stage
 
 cudaError_t launch_gemm(const GemmArgs& a, cudaStream_t stream);
 cudaError_t gemm_init();            // one-time: opt in to large dynamic shared memory
+cudaError_t launch_gemm_pair(const GemmArgs& a, cudaStream_t stream);
+cudaError_t gemm_pair_init();
 
 }  // namespace mx
