@@ -4,8 +4,12 @@
 // 1-CTA kernel (gemm.cu) is bound by exactly that operand traffic.  Each CTA keeps the accumulator of its own 128
 // rows (all 256 columns) in its TMEM.
 //
-// Roles per CTA (10 warps), all waits bounded as in gemm.cu:
-//   warp 0      TMA producer: own A rows, own half of B (completion counted on the LEADER's barrier), own scale tiles;
+// The scale tiles travel in their own, deeper ring (8 slots, decoupled from the 6 operand stages), so they are in
+// TMEM long before the MMAs that need them; the only tight loop left is the reuse of an operand stage.
+//
+// Roles per CTA (11 warps), all waits bounded as in gemm.cu:
+//   warp 0      TMA producer: own A rows, own half of B (completion counted on the LEADER's barrier);
+//   warp 10     scale loader: own A-row scale tiles and the scale tiles of all 256 B rows, bulk copies into the ring;
 //   warp 1      MMA issuer, leader CTA only: four K = 64 pair-MMAs per stage; tcgen05.commit frees stage, scale slot
 //               and accumulator in BOTH CTAs;
 //   warps 2..5  epilogue of the CTA's own 128 x 256 half tile;
@@ -25,12 +29,14 @@ constexpr uint32_t kAB = 128 * kGemmBKBytes;                // 16 KB: 128 rows x
 constexpr uint32_t kSfTile = 512;
 constexpr uint32_t kSfaB = 2 * kSfTile;                     // own 128 A rows, 2 tiles (8 K-blocks) per stage
 constexpr uint32_t kSfbB = 2 * 2 * kSfTile;                 // all 256 B rows
-constexpr uint32_t kStageB = 2 * kAB + kSfaB + kSfbB;       // 35 KB, multiple of 1024
-constexpr uint32_t kSmemP = kStagesP * kStageB + 1024 + 512;
+constexpr uint32_t kStageB = 2 * kAB;                       // 32 KB: A rows + B half
+constexpr int kSfSlotsP = kStagesP;                         // scale ring: shared-memory slot i feeds TMEM slot i; same ring
+                                                            // index as the operand stages so ONE commit frees both
+constexpr uint32_t kSfSlotB = kSfaB + kSfbB;                // 3 KB
+constexpr uint32_t kSmemP = kStagesP * kStageB + kSfSlotsP * kSfSlotB + 1024 + 512;
 constexpr uint32_t kAccColP = 0, kSfColP = 256, kSfSlotColsP = 24;
-constexpr int kSfSlotsP = 4;
 constexpr int kGroupMP = 8;                                 // rasterisation: 8 pair-tiles (2048 rows) share B tiles in L2
-constexpr int kThreadsP = 10 * 32;
+constexpr int kThreadsP = 11 * 32;
 
 struct ParamsP {
     const uint8_t* sfa;
@@ -56,11 +62,12 @@ __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(kThreadsP, 1)
 gemm_mxf4_pair_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant__ CUtensorMap tmap_b, const ParamsP p) {
     extern __shared__ uint8_t smem_raw[];
     uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
-    uint64_t* bars = reinterpret_cast<uint64_t*>(smem + kStagesP * kStageB);
+    uint8_t* sf_ring = smem + kStagesP * kStageB;
+    uint64_t* bars = reinterpret_cast<uint64_t*>(sf_ring + kSfSlotsP * kSfSlotB);
     uint64_t* full_bar = bars;                              // [kStagesP] leader: A and B halves of both CTAs landed
     uint64_t* empty_bar = full_bar + kStagesP;              // [kStagesP] per CTA: stage free (pair commit)
-    uint64_t* sfl_full = empty_bar + kStagesP;              // [kStagesP] per CTA: own scale tiles landed
-    uint64_t* sf_full = sfl_full + kStagesP;                // [kSfSlotsP] leader: scales of both CTAs are in TMEM
+    uint64_t* sfl_full = empty_bar + kStagesP;              // [kSfSlotsP] per CTA: scale tiles landed in the ring slot
+    uint64_t* sf_full = sfl_full + kSfSlotsP;                // [kSfSlotsP] leader: scales of both CTAs are in TMEM
     uint64_t* sf_empty = sf_full + kSfSlotsP;               // [kSfSlotsP] per CTA: scale slot free (pair commit)
     uint64_t* tmem_full = sf_empty + kSfSlotsP;             // per CTA: accumulator complete (pair commit)
     uint64_t* tmem_empty = tmem_full + 1;                   // leader: both CTAs drained their accumulators
@@ -77,8 +84,8 @@ gemm_mxf4_pair_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_c
     const uint32_t total = my_tiles * (uint32_t)num_kt;
 
     if (threadIdx.x == 0) {
-        for (int s = 0; s < kStagesP; ++s) { mbar_init(&full_bar[s], 1); mbar_init(&empty_bar[s], 1); mbar_init(&sfl_full[s], 1); }
-        for (int s = 0; s < kSfSlotsP; ++s) { mbar_init(&sf_full[s], 8); mbar_init(&sf_empty[s], 1); }
+        for (int s = 0; s < kStagesP; ++s) { mbar_init(&full_bar[s], 1); mbar_init(&empty_bar[s], 1); }
+        for (int s = 0; s < kSfSlotsP; ++s) { mbar_init(&sfl_full[s], 1); mbar_init(&sf_full[s], 8); mbar_init(&sf_empty[s], 1); }
         mbar_init(tmem_full, 1);
         mbar_init(tmem_empty, 8);
         *abort_flag = 0;
@@ -105,23 +112,13 @@ gemm_mxf4_pair_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_c
                 int mt, nt;
                 tile_coords_p((int)(pair + tl * num_pairs), p.m_tiles, p.n_tiles, mt, nt);
                 const int a_rt = 2 * mt + (int)rank;                            // this CTA's 128-row tile of A
-                const bool has_a = (int64_t)a_rt * 128 < p.M;
-                const int n_row_tiles = min(2, (int)((p.N - (int64_t)nt * PN + 127) >> 7));
                 for (int kt = 0; kt < num_kt; ++kt, ++it) {
                     const int s = it % kStagesP;
                     if (!(ok = mbar_wait(&empty_bar[s], ((it / kStagesP) & 1) ^ 1, abort_flag))) break;
                     uint8_t* st = smem + s * kStageB;
-                    const int nch = min(2, nkc - 2 * kt);
                     if (rank == 0) mbar_expect_tx(&full_bar[s], 4 * kAB);       // two loads from each CTA
                     tma_load_2d_pair(st, &tmap_a, &full_bar[s], kt * kGemmBKBytes, a_rt * 128);
                     tma_load_2d_pair(st + kAB, &tmap_b, &full_bar[s], kt * kGemmBKBytes, nt * PN + (int)rank * 128);
-                    const uint32_t sf_bytes = (uint32_t)nch * kSfTile * ((has_a ? 1u : 0u) + (uint32_t)n_row_tiles);
-                    if (sf_bytes != 0) mbar_expect_tx(&sfl_full[s], sf_bytes); else mbar_arrive(&sfl_full[s]);
-                    if (has_a)
-                        bulk_load(st + 2 * kAB, p.sfa + ((int64_t)a_rt * nkc + 2 * kt) * kSfTile, nch * kSfTile, &sfl_full[s]);
-                    for (int j = 0; j < n_row_tiles; ++j)
-                        bulk_load(st + 2 * kAB + kSfaB + j * 2 * kSfTile,
-                                  p.sfb + ((int64_t)(nt * 2 + j) * nkc + 2 * kt) * kSfTile, nch * kSfTile, &sfl_full[s]);
                 }
             }
             if (!ok) *abort_flag = 1;
@@ -154,25 +151,49 @@ gemm_mxf4_pair_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_c
                                      (sfa_t + 4 * (kb >> 1)) | (sf_id << 30), (sfb_t + 8 * (kb >> 1)) | (sf_id << 30),
                                      (kt | kb) != 0 ? 1u : 0u);
                 }
-                tc_commit_pair(&empty_bar[s]);
-                tc_commit_pair(&sf_empty[slot]);
+                tc_commit_pair(&empty_bar[s]);                                 // frees the operand stage and the scale slot
                 if (kt == num_kt - 1) { tc_commit_pair(tmem_full); ++tile_i; }
             }
             if (!ok) *abort_flag = 1;
         }
+    } else if (warp == 10) {
+        // ------------------------------------------------------------------ scale loader (both CTAs)
+        if (lane == 0) {
+            uint32_t it = 0;
+            bool ok = true;
+            for (uint32_t tl = 0; tl < my_tiles && ok; ++tl) {
+                int mt, nt;
+                tile_coords_p((int)(pair + tl * num_pairs), p.m_tiles, p.n_tiles, mt, nt);
+                const int a_rt = 2 * mt + (int)rank;
+                const bool has_a = (int64_t)a_rt * 128 < p.M;
+                const int n_row_tiles = min(2, (int)((p.N - (int64_t)nt * PN + 127) >> 7));
+                for (int kt = 0; kt < num_kt; ++kt, ++it) {
+                    const int slot = it % kSfSlotsP;
+                    // the slot's previous scales (shared memory and TMEM) are dead once the MMAs that read them completed
+                    if (!(ok = mbar_wait(&empty_bar[slot], ((it / kSfSlotsP) & 1) ^ 1, abort_flag))) break;
+                    uint8_t* dst = sf_ring + slot * kSfSlotB;
+                    const int nch = min(2, nkc - 2 * kt);
+                    mbar_expect_tx(&sfl_full[slot], (uint32_t)nch * kSfTile * ((has_a ? 1u : 0u) + (uint32_t)n_row_tiles));
+                    if (has_a) bulk_load(dst, p.sfa + ((int64_t)a_rt * nkc + 2 * kt) * kSfTile, nch * kSfTile, &sfl_full[slot]);
+                    for (int j = 0; j < n_row_tiles; ++j)
+                        bulk_load(dst + kSfaB + j * 2 * kSfTile, p.sfb + ((int64_t)(nt * 2 + j) * nkc + 2 * kt) * kSfTile,
+                                  nch * kSfTile, &sfl_full[slot]);
+                }
+            }
+            if (!ok) *abort_flag = 1;
+        }
     } else if (warp >= 6) {
-        // ------------------------------------------------------------------ scale movers (both CTAs)
+        // ------------------------------------------------------------------ scale movers (both CTAs, warps 6..9)
         const int q = warp & 3;
         const uint32_t lane_base = (uint32_t)(q * 32) << 16;
         bool ok = true;
         for (uint32_t it = 0; it < total; ++it) {
-            const int s = it % kStagesP, slot = it % kSfSlotsP;
-            ok = mbar_wait(&sf_empty[slot], ((it / kSfSlotsP) & 1) ^ 1, abort_flag) &&
-                 mbar_wait(&sfl_full[s], (it / kStagesP) & 1, abort_flag);
-            ok = __all_sync(0xffffffffu, ok);
+            const int slot = it % kSfSlotsP;
+            if (lane == 0) ok = mbar_wait(&sfl_full[slot], (it / kSfSlotsP) & 1, abort_flag);
+            ok = __shfl_sync(0xffffffffu, ok, 0);
             if (!ok) break;
             tc_fence_after_sync();
-            const uint4* sf = reinterpret_cast<const uint4*>(smem + s * kStageB + 2 * kAB) + lane;       // 32 uint4 per tile
+            const uint4* sf = reinterpret_cast<const uint4*>(sf_ring + slot * kSfSlotB) + lane;          // 32 uint4 per tile
             const uint32_t sfa_t = tmem_base + lane_base + kSfColP + slot * kSfSlotColsP, sfb_t = sfa_t + 8;
             tmem_st_32x32b_x8(sfa_t, sf[0], sf[32]);
             tmem_st_32x32b_x16(sfb_t, sf[64], sf[128], sf[96], sf[160]);
@@ -189,8 +210,8 @@ gemm_mxf4_pair_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_c
         for (uint32_t tl = 0; tl < my_tiles; ++tl) {
             int mt, nt;
             tile_coords_p((int)(pair + tl * num_pairs), p.m_tiles, p.n_tiles, mt, nt);
-            ok = mbar_wait(tmem_full, tl & 1, abort_flag);
-            ok = __all_sync(0xffffffffu, ok);
+            if (lane == 0) ok = mbar_wait(tmem_full, tl & 1, abort_flag);
+            ok = __shfl_sync(0xffffffffu, ok, 0);
             if (!ok) break;
             tc_fence_after_sync();
             const int64_t row = (int64_t)mt * PM + (int64_t)rank * 128 + q * 32 + lane;

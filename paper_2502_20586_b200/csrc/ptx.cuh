@@ -72,7 +72,7 @@ __device__ __forceinline__ bool mbar_try_wait_hint(uint64_t* bar, uint32_t parit
 static __device__ __noinline__ bool mbar_wait_slow(uint64_t* bar, uint32_t parity, const volatile uint32_t* abort) {
     const uint64_t t0 = global_timer_ns();
     for (uint32_t i = 0;; ++i) {
-        if (mbar_try_wait_hint(bar, parity, 2000u)) return true;
+        if (mbar_try_wait_hint(bar, parity, 1000u)) return true;
         if (abort != nullptr && *abort != 0u) return false;
         if ((i & 15u) == 15u && global_timer_ns() - t0 > kWaitLimitNs) break;
     }
