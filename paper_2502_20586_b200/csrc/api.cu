@@ -23,7 +23,7 @@ struct Runtime {
     std::once_flag once;
     mxfp4_status status = MXFP4_OK;
     EncodeTiledFn encode = nullptr;
-    bool gemm_pair = true;       // CTA-pair GEMM unless MXFP4_GEMM_1CTA=1 (debugging / comparison)
+    bool gemm_pair = false;      // CTA-pair GEMM (gemm_pair.cu) only with MXFP4_GEMM_PAIR=1: measured slightly slower
 };
 Runtime g_rt;
 
@@ -48,8 +48,8 @@ mxfp4_status runtime_init() {
         }
         g_rt.encode = reinterpret_cast<EncodeTiledFn>(fn);
         if (mx::gemm_init() != cudaSuccess || mx::gemm_pair_init() != cudaSuccess || mx::quant_tc_init() != cudaSuccess) g_rt.status = MXFP4_ERR_CUDA;
-        const char* one_cta = getenv("MXFP4_GEMM_1CTA");
-        g_rt.gemm_pair = !(one_cta != nullptr && one_cta[0] == '1');
+        const char* pair = getenv("MXFP4_GEMM_PAIR");
+        g_rt.gemm_pair = pair != nullptr && pair[0] == '1';
     });
     return g_rt.status;
 }

@@ -37,7 +37,7 @@ constexpr uint32_t kTmemCols = 512;
 constexpr uint32_t kAccCol = 0;                             // 256 fp32 accumulator columns
 constexpr uint32_t kSfCol = 256;                            // kSfSlots slots of (8 SFA + 16 SFB) columns
 constexpr uint32_t kSfSlotCols = 24;
-constexpr int kSfSlots = 4;
+constexpr int kSfSlots = kStages;                           // scale slot i belongs to stage i: one commit frees both
 constexpr int kGroupM = 16;                                 // tile rasterisation: 16 m-tiles share B tiles in L2
 constexpr int kThreads = 10 * 32;
 
@@ -69,8 +69,7 @@ gemm_mxf4_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_consta
     uint64_t* full_bar = bars;                              // [kStages]  TMA -> MMA, scale movers
     uint64_t* empty_bar = full_bar + kStages;               // [kStages]  MMA -> TMA
     uint64_t* sf_full = empty_bar + kStages;                // [kSfSlots] scale movers -> MMA
-    uint64_t* sf_empty = sf_full + kSfSlots;                // [kSfSlots] MMA -> scale movers
-    uint64_t* tmem_full = sf_empty + kSfSlots;              // MMA -> epilogue
+    uint64_t* tmem_full = sf_full + kSfSlots;               // MMA -> epilogue
     uint64_t* tmem_empty = tmem_full + 1;                   // epilogue -> MMA
     uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(tmem_empty + 1);
     volatile uint32_t* abort_flag = tmem_slot + 1;
@@ -84,7 +83,7 @@ gemm_mxf4_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_consta
 
     if (threadIdx.x == 0) {
         for (int s = 0; s < kStages; ++s) { mbar_init(&full_bar[s], 1); mbar_init(&empty_bar[s], 1); }
-        for (int s = 0; s < kSfSlots; ++s) { mbar_init(&sf_full[s], 4); mbar_init(&sf_empty[s], 1); }
+        for (int s = 0; s < kSfSlots; ++s) mbar_init(&sf_full[s], 4);
         mbar_init(tmem_full, 1);
         mbar_init(tmem_empty, 4);
         *abort_flag = 0;
@@ -155,8 +154,7 @@ gemm_mxf4_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_consta
                                 (sfa_t + 4 * (kb >> 1)) | (sf_id << 30), (sfb_t + 8 * (kb >> 1)) | (sf_id << 30),
                                 (kt | kb) != 0 ? 1u : 0u);
                 }
-                tc_commit(&empty_bar[s]);                                     // stage and scale slot are free once
-                tc_commit(&sf_empty[slot]);                                   // these MMAs have read them
+                tc_commit(&empty_bar[s]);                // one commit frees the stage and its scale slot (same ring index)
                 if (kt == num_kt - 1) { tc_commit(tmem_full); ++tile_i; }
             }
             if (!ok) *abort_flag = 1;
@@ -172,8 +170,7 @@ gemm_mxf4_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_consta
         bool ok = true;
         for (uint32_t it = 0; it < total; ++it) {
             const int s = it % kStages, slot = it % kSfSlots;
-            ok = mbar_wait(&sf_empty[slot], ((it / kSfSlots) & 1) ^ 1, abort_flag) &&
-                 mbar_wait(&full_bar[s], (it / kStages) & 1, abort_flag);
+            ok = mbar_wait(&full_bar[s], (it / kStages) & 1, abort_flag);
             ok = __all_sync(0xffffffffu, ok);
             if (!ok) break;
             tc_fence_after_sync();
