@@ -35,6 +35,9 @@ UNIT = "TFLOP/s"
 NOMINAL_FP4_TFLOPS = 9000.0          # dense, NVIDIA's figure; context only
 BF16_TO_FP4 = 4.0                    # nominal dense ratio 9 / 2.25 PFLOP/s
 QUANT_BYTES_PER_ELEM = 2.0 + 0.5 + 1.0 / 32.0   # bf16 in, E2M1 code + E8M0 scale out
+# DRAM bytes moved / algorithmic bytes of the GEMM, from one ncu capture (profiles/gemm_mxf4_16384x4096x16384.md:
+# 453.5 MB measured against 312.6 MB of codes, scales and bf16 output); applied to the average launch of the step.
+GEMM_TRAFFIC_OVER_ALGORITHMIC = 1.45
 
 
 def load_peaks():
@@ -278,6 +281,8 @@ def run_gpu(args):
             d = agg.setdefault(kind, [0.0, 0.0, 0])
             d[0] += a.elapsed_time(b) * 1e-3; d[1] += work; d[2] += 1
         gemm_t, gemm_fl, gemm_n = agg["gemm"]
+        gemm_bytes = k_roof * sum((l.b * l.m + l.n * l.m) * 0.53125 + l.b * l.n * 2 + (l.m * l.b + l.n * l.b) * 0.53125 + l.m * l.n * 2
+                                  for l in layers)
         gemm_tflops = gemm_fl / gemm_t / 1e12
         kernels = {}
         for kind in ("quant_row", "quant_tr"):
@@ -349,7 +354,9 @@ def run_gpu(args):
             "clocks": clocks,
             "roofline": None if gemm_tflops is None else {
                          "kernel": "gemm_mxf4_kernel", "bound": "tensor", "achieved": gemm_tflops, "peak": fp4_peak, "unit": "TFLOP/s",
-                         "frac": gemm_tflops / fp4_peak, "traffic": None,
+                         "frac": gemm_tflops / fp4_peak,
+                         "traffic": GEMM_TRAFFIC_OVER_ALGORITHMIC * gemm_bytes / gemm_n,
+                         "traffic_note": "bytes per average launch = algorithmic bytes x 1.45 (ratio from an ncu capture of the 16384x4096x16384 launch)",
                          "peak_source": f"4 x {peaks['source']} sustained bf16 ({peaks['bf16_sustained']} TFLOP/s); no FP4 peak was measured"},
             "kernels": kernels,
             "hbm_peak_gbs": peaks["hbm_gbs"], "peaks_source": peaks["source"],
