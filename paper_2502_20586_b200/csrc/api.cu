@@ -237,9 +237,16 @@ mxfp4_status mxfp4_linear_backward(const void* dY, const void* X, const void* W,
         {dY, b, m, m, 0, g, rounding, seed, 3u, c[2], s[2], 1, nullptr},   // dY^T [m, K = b]
         {X, b, n, n, 0, g, rounding, seed, 4u, c[3], s[3], 1, nullptr},    // X^T  [n, K = b]
     };
+    bool all_tc = true;
     for (int i = 0; i < 4; ++i) {
         attach_input_map(q[i]);
-        if (mx::launch_quantize(q[i], stream) != cudaSuccess) return MXFP4_ERR_CUDA;
+        all_tc = all_tc && mx::quant_tc_eligible(q[i]);
+    }
+    if (all_tc) {                                   // the four views of the call in one launch
+        if (mx::launch_quantize_tc_group(q, 4, false, stream) != cudaSuccess) return MXFP4_ERR_CUDA;
+    } else {
+        for (int i = 0; i < 4; ++i)
+            if (mx::launch_quantize(q[i], stream) != cudaSuccess) return MXFP4_ERR_CUDA;
     }
     // lines 7-11: two MXFP4 GEMMs; the 16/9 un-does the two 3/4 pre-scales of Algorithm 2.
     const float alpha = rounding == MXFP4_ROUND_SR ? 16.0f / 9.0f : 1.0f;

@@ -26,6 +26,9 @@ struct QuantArgs {
 bool quant_tc_eligible(const QuantArgs& a);
 cudaError_t quant_tc_init();
 cudaError_t launch_quantize_tc(const QuantArgs& a, bool dump_y, cudaStream_t stream);
+// Up to kQuantMaxViews eligible views sharing g, seed, rounding and scale layout, in ONE launch.
+constexpr int kQuantMaxViews = 4;
+cudaError_t launch_quantize_tc_group(const QuantArgs* a, int n, bool dump_y, cudaStream_t stream);
 
 cudaError_t launch_quantize(const QuantArgs& a, cudaStream_t stream);
 cudaError_t launch_rht_dump(const QuantArgs& a, cudaStream_t stream);

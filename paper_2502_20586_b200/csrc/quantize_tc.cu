@@ -11,6 +11,10 @@
 // views (W, dY^T, X^T of Algorithm 3) the very same TMA tile is handed to the MMA as an MN-major operand, so the
 // transposition costs nothing.
 //
+// One launch can quantise up to four operand views that share g, seed and rounding (the four views of one
+// backward call, Algorithm 3 lines 3-6): their tiles form one list that the persistent CTAs walk, which removes
+// three launch / prologue / drain gaps per layer.
+//
 //   warp 0        TMA producer (two 64-column x 128-row boxes per tile, 128-byte swizzle, 4-stage ring)
 //   warp 1        MMA issuer (8 K=16 MMAs per tile into one of four 128-column TMEM accumulators)
 //   warps 2..17   epilogue, two groups of eight warps on alternate tiles: warp = (TMEM lane quadrant, 64 columns):
@@ -35,23 +39,33 @@ constexpr int kAccBufs = 4;                         // 4 x 128 TMEM columns
 constexpr int kEpiWarps = 16;
 constexpr int kThreadsQ = (2 + kEpiWarps) * 32;
 
-struct QParams {
-    int64_t R, K;              // output operand [R, K]
-    int64_t r_tiles, k_tiles;
-    int reduce_dim, g, rounding;
-    uint64_t seed;
+struct QView {                 // one operand view: output operand [R, K] read from x [rows, cols]
+    int64_t R, K;
+    uint32_t r_tiles, k_tiles;
+    uint32_t tile_begin;       // first index of this view in the launch's tile list
+    int reduce_dim;            // 1: K runs along x columns (x tile is the K-major operand); 0: along x rows (MN-major)
     uint32_t stream_tag;
     uint8_t* codes;
     uint8_t* scales;
-    int sf_native;
-    float* y_out;
-    PipeConsts pipe;          // see quant_math.cuh: constants kept opaque to the compiler
-    PhiloxKeys keys;          // the ten Philox round keys of `seed` (key schedule only; the rounds run on the device)
+    float* y_out;              // transform dump only
+};
+
+struct QParams {
+    QView view[kQuantMaxViews];
+    int n_views;
+    uint32_t n_tiles;          // over all views
+    int g, sf_native;
+    uint64_t seed;
+    PipeConsts pipe;           // see quant_math.cuh: constants kept opaque to the compiler
+    PhiloxKeys keys;           // the ten Philox round keys of `seed` (key schedule only; the rounds run on the device)
+};
+
+struct QMaps {
+    CUtensorMap x[kQuantMaxViews];
 };
 
 // bf16 entry (n, k) of the transform operand, stored N x K (K-major): T[k][n] = S_k H_g[k][n] inside a g-chunk.
 __device__ __forceinline__ uint32_t transform_entry(int n, int k, int g, const uint32_t (&sign)[4]) {
-    if (g == 0) return n == k ? 0x3F80u : 0u;
     if ((n ^ k) & ~(g - 1)) return 0u;                                   // different g-chunks
     const int kk = k & (g - 1);
     const uint32_t neg = ((sign[kk >> 5] >> (kk & 31)) ^ (uint32_t)__popc(k & n & (g - 1))) & 1u;
@@ -59,11 +73,31 @@ __device__ __forceinline__ uint32_t transform_entry(int n, int k, int g, const u
     return mag | (neg << 15);
 }
 
+// Position of a tile in the launch's list: its view and its (row tile, k tile) there.  Tiles of a view with a
+// contiguous reduce dimension run along k first, the transposing ones along the output rows first, so that CTAs
+// working side by side read neighbouring 256-byte row segments of x.
+struct TilePos {
+    int v;
+    uint32_t rt, kt;
+};
+__device__ __forceinline__ TilePos locate_tile(const QParams& p, uint32_t t) {
+    int v = 0;
+#pragma unroll
+    for (int i = 1; i < kQuantMaxViews; ++i)
+        if (i < p.n_views && t >= p.view[i].tile_begin) v = i;
+    const uint32_t local = t - p.view[v].tile_begin;
+    TilePos pos;
+    pos.v = v;
+    if (p.view[v].reduce_dim == 1) { pos.rt = local / p.view[v].k_tiles; pos.kt = local - pos.rt * p.view[v].k_tiles; }
+    else { pos.kt = local / p.view[v].r_tiles; pos.rt = local - pos.kt * p.view[v].r_tiles; }
+    return pos;
+}
+
 enum { kModeSR = 0, kModeRN = 1, kModeDump = 2 };
 
 template <int MODE>
 __global__ void __launch_bounds__(kThreadsQ, 1)
-quantize_tc_kernel(const __grid_constant__ CUtensorMap tmap_x, const QParams p) {
+quantize_tc_kernel(const __grid_constant__ QMaps maps, const __grid_constant__ QParams p) {
     extern __shared__ uint8_t smem_raw[];
     uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
     uint8_t* smem_t = smem + kStagesQ * kTileBytes;
@@ -76,14 +110,14 @@ quantize_tc_kernel(const __grid_constant__ CUtensorMap tmap_x, const QParams p) 
     volatile uint32_t* abort_flag = tmem_slot + 1;
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-    const int64_t num_tiles = p.r_tiles * p.k_tiles;
+    const uint32_t num_tiles = p.n_tiles;
 
     if (threadIdx.x == 0) {
         for (int s = 0; s < kStagesQ; ++s) { mbar_init(&full_bar[s], 1); mbar_init(&empty_bar[s], 1); }
         for (int b = 0; b < kAccBufs; ++b) { mbar_init(&acc_full[b], 1); mbar_init(&acc_empty[b], kEpiWarps / 2); }
         *abort_flag = 0;
         mbar_fence_init();
-        prefetch_tensormap(&tmap_x);
+        for (int v = 0; v < p.n_views; ++v) prefetch_tensormap(&maps.x[v]);
     }
     if (warp == 1) {
         tmem_alloc(tmem_slot, 512);
@@ -92,11 +126,8 @@ quantize_tc_kernel(const __grid_constant__ CUtensorMap tmap_x, const QParams p) 
     {
         // Transform operand, written in the 128-byte-swizzled K-major layout the MMA descriptor expects:
         // entry (n, k) at box (k / 64), row n (128 B pitch), 16-byte chunk ((k % 64) / 8) ^ (n % 8).
-        uint32_t sign[4] = {0u, 0u, 0u, 0u};
-        if (p.g != 0) {
-            const uint4 o = philox4x32_10(0u, 0u, 0u, 0u, (uint32_t)p.seed, (uint32_t)(p.seed >> 32));
-            sign[0] = o.x; sign[1] = o.y; sign[2] = o.z; sign[3] = o.w;
-        }
+        const uint4 o = philox4x32_10(0u, 0u, 0u, 0u, (uint32_t)p.seed, (uint32_t)(p.seed >> 32));
+        const uint32_t sign[4] = {o.x, o.y, o.z, o.w};
         for (int task = threadIdx.x; task < 128 * 16; task += kThreadsQ) {
             const int n = task >> 4, c = task & 15;                      // c: 16-byte chunk = 8 consecutive k
             uint32_t w[4];
@@ -118,22 +149,17 @@ quantize_tc_kernel(const __grid_constant__ CUtensorMap tmap_x, const QParams p) 
         if (lane == 0) {
             uint32_t it = 0;
             bool ok = true;
-            for (int64_t t = blockIdx.x; t < num_tiles; t += gridDim.x, ++it) {
+            for (uint32_t t = blockIdx.x; t < num_tiles; t += gridDim.x, ++it) {
                 const int s = it % kStagesQ;
                 if (!(ok = mbar_wait(&empty_bar[s], ((it / kStagesQ) & 1) ^ 1, abort_flag))) break;
-                // tile -> (row tile of the OUTPUT operand, k tile); x coordinates depend on the access pattern
-                int32_t cx, cy;
-                if (p.reduce_dim == 1) {            // output rows = x rows; k = x columns; consecutive tiles along k
-                    const int64_t rt = t / p.k_tiles, kt = t - rt * p.k_tiles;
-                    cx = (int32_t)(kt * kTile); cy = (int32_t)(rt * kTile);
-                } else {                            // output rows = x columns; k = x rows; consecutive tiles along x columns
-                    const int64_t kt = t / p.r_tiles, rt = t - kt * p.r_tiles;
-                    cx = (int32_t)(rt * kTile); cy = (int32_t)(kt * kTile);
-                }
+                const TilePos pos = locate_tile(p, t);
+                // x coordinates: (column, row).  reduce_dim 1: output rows = x rows, k = x columns; else swapped.
+                const bool rowwise = p.view[pos.v].reduce_dim == 1;
+                const int32_t cx = (int32_t)((rowwise ? pos.kt : pos.rt) * kTile), cy = (int32_t)((rowwise ? pos.rt : pos.kt) * kTile);
                 uint8_t* st = smem + s * kTileBytes;
                 mbar_expect_tx(&full_bar[s], kTileBytes);
-                tma_load_2d(st, &tmap_x, &full_bar[s], cx, cy);
-                tma_load_2d(st + kBoxBytes, &tmap_x, &full_bar[s], cx + 64, cy);
+                tma_load_2d(st, &maps.x[pos.v], &full_bar[s], cx, cy);
+                tma_load_2d(st + kBoxBytes, &maps.x[pos.v], &full_bar[s], cx + 64, cy);
             }
             if (!ok) *abort_flag = 1;
         }
@@ -142,13 +168,18 @@ quantize_tc_kernel(const __grid_constant__ CUtensorMap tmap_x, const QParams p) 
         if (lane == 0) {
             // kind::f16 instruction descriptor: D = fp32 (bits 4-5 = 1), A = B = bf16 (bits 7-9, 10-12 = 1),
             // A major at bit 15 (0 = K-major, 1 = MN-major), B K-major, N >> 3 at bit 17, M >> 4 at bit 24.
-            const uint32_t idesc = (1u << 4) | (1u << 7) | (1u << 10) | ((p.reduce_dim == 0 ? 1u : 0u) << 15) |
-                                   ((uint32_t)(kTile >> 3) << 17) | ((uint32_t)(kTile >> 4) << 24);
+            const uint32_t idesc_k = (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(kTile >> 3) << 17) | ((uint32_t)(kTile >> 4) << 24);
             const uint32_t t_addr = smem_u32(smem_t);
             uint32_t it = 0;
             bool ok = true;
-            for (int64_t t = blockIdx.x; t < num_tiles; t += gridDim.x, ++it) {
+            for (uint32_t t = blockIdx.x; t < num_tiles; t += gridDim.x, ++it) {
                 const int s = it % kStagesQ, b = it % kAccBufs;
+                int v = 0;
+#pragma unroll
+                for (int i = 1; i < kQuantMaxViews; ++i)
+                    if (i < p.n_views && t >= p.view[i].tile_begin) v = i;
+                const bool rowwise = p.view[v].reduce_dim == 1;
+                const uint32_t idesc = idesc_k | ((rowwise ? 0u : 1u) << 15);
                 if (!(ok = mbar_wait(&acc_empty[b], ((it / kAccBufs) & 1) ^ 1, abort_flag))) break;
                 if (!(ok = mbar_wait(&full_bar[s], (it / kStagesQ) & 1, abort_flag))) break;
                 tc_fence_after_sync();
@@ -156,7 +187,7 @@ quantize_tc_kernel(const __grid_constant__ CUtensorMap tmap_x, const QParams p) 
 #pragma unroll
                 for (int ks = 0; ks < 8; ++ks) {                           // K = 16 per MMA
                     uint64_t adesc;
-                    if (p.reduce_dim == 1)      // K-major: box ks/4, 32 bytes of K per step inside the 128-byte swizzle atom
+                    if (rowwise)                // K-major: box ks/4, 32 bytes of K per step inside the 128-byte swizzle atom
                         adesc = make_smem_desc(a_addr + (ks >> 2) * kBoxBytes + (ks & 3) * 32, 16, 1024, 2);
                     else                        // MN-major: 16 k-rows of 128 B per step; the second 64 output rows sit one box further
                         adesc = make_smem_desc(a_addr + ks * 2048, kBoxBytes, 1024, 2);
@@ -179,41 +210,41 @@ quantize_tc_kernel(const __grid_constant__ CUtensorMap tmap_x, const QParams p) 
         const int grp = e >> 3;
         const int half = (e >> 2) & 1;
         const float cg = p.g == 32 ? 0.17677669529663687f : p.g == 128 ? 0.08838834764831845f : 1.0f;
-        const uint32_t k_tiles = (uint32_t)p.k_tiles, r_tiles = (uint32_t)p.r_tiles;
-        const uint32_t nkb = (uint32_t)(p.K >> 5), nkc = (nkb + 3) >> 2;
-        const uint32_t ntile = (uint32_t)num_tiles, stride = 2u * gridDim.x;
+        const uint32_t stride = 2u * gridDim.x;
         const uint32_t lane_row = (uint32_t)(q * 32 + lane);
         bool ok = true;
 
-        // Tile t -> (row tile, k tile) of the output operand; t advances by `stride` per iteration, so the
-        // coordinates are carried along instead of divided out each time.
-        const bool rowwise = p.reduce_dim == 1;
-        const uint32_t fast = rowwise ? k_tiles : r_tiles;                    // extent of the fast-running coordinate
-        const uint32_t dq = stride / fast, dr = stride - dq * fast;
-        const uint64_t K64 = (uint64_t)p.K;
-        auto first_elem = [&](uint32_t rt, uint32_t kt) -> uint64_t {        // linear index of this thread's first element
-            return (uint64_t)(rt * (uint32_t)kTile + lane_row) * K64 + (uint64_t)(kt * (uint32_t)kTile + (uint32_t)half * 64u);
+        auto first_elem = [&](const TilePos& pos) -> uint64_t {          // linear index of this thread's first element
+            return (uint64_t)(pos.rt * (uint32_t)kTile + lane_row) * (uint64_t)p.view[pos.v].K +
+                   (uint64_t)(pos.kt * (uint32_t)kTile + (uint32_t)half * 64u);
         };
 
         uint32_t it = (uint32_t)grp;
         uint32_t t = blockIdx.x + it * gridDim.x;
-        uint32_t slow_c = t / fast, fast_c = t - slow_c * fast;               // one division per thread
+        TilePos pos = locate_tile(p, t < num_tiles ? t : 0u);
         uint32_t rw0[8], rw1[8];
         if (MODE == kModeSR) {
-            const uint64_t i0 = rowwise ? first_elem(slow_c, fast_c) : first_elem(fast_c, slow_c);
-            sr_draws32(p.keys, p.stream_tag, i0, rw0);
-            sr_draws32(p.keys, p.stream_tag, i0 + 32, rw1);
+            const uint64_t i0 = first_elem(pos);
+            sr_draws32(p.keys, p.view[pos.v].stream_tag, i0, rw0);
+            sr_draws32(p.keys, p.view[pos.v].stream_tag, i0 + 32, rw1);
         }
-        for (; t < ntile; t += stride, it += 2) {
+        for (; t < num_tiles; t += stride, it += 2) {
             const int b = it % kAccBufs;
-            const uint32_t rt = rowwise ? slow_c : fast_c, kt = rowwise ? fast_c : slow_c;
-            fast_c += dr; slow_c += dq;
-            if (fast_c >= fast) { fast_c -= fast; ++slow_c; }                  // coordinates of tile t + stride
+            const QView& vw = p.view[pos.v];
+            const uint32_t rt = pos.rt, kt = pos.kt;
+            const int64_t K = vw.K;
             const int64_t row = (int64_t)rt * kTile + lane_row;                 // output row
             const int64_t k0 = (int64_t)kt * kTile + half * 64;
-            const bool live = row < p.R;
-            // draws of the next tile of this group (computed even past the end: they are simply not used)
-            const uint64_t i_next = rowwise ? first_elem(slow_c, fast_c) : first_elem(fast_c, slow_c);
+            const bool live = row < vw.R;
+            uint8_t* code_dst = vw.codes + row * (K >> 1) + (k0 >> 1);
+            const uint32_t nkb = (uint32_t)(K >> 5), nkc = (nkb + 3) >> 2;
+            uint8_t* scale_dst = vw.scales + (p.sf_native ? ((int64_t)(rt * nkc + kt) * 512 + lane * 16 + q * 4 + half * 2)
+                                                           : row * nkb + (k0 >> 5));
+            float* y_dst = MODE == kModeDump ? vw.y_out + row * K + k0 : nullptr;
+            // position and draws of the next tile of this group (past the end: computed but not used)
+            pos = locate_tile(p, t + stride < num_tiles ? t + stride : 0u);
+            const uint64_t i_next = first_elem(pos);
+            const uint32_t tag_next = p.view[pos.v].stream_tag;
             ok = mbar_wait(&acc_full[b], (it / kAccBufs) & 1, abort_flag);
             ok = __all_sync(0xffffffffu, ok);
             if (!ok) break;
@@ -221,16 +252,15 @@ quantize_tc_kernel(const __grid_constant__ CUtensorMap tmap_x, const QParams p) 
             const uint32_t taddr = tmem_base + ((uint32_t)(q * 32) << 16) + b * kTile + half * 64;
             uint32_t raw[32], n0[8], n1[8], packed[4], sb0 = 0, sb1 = 0;
             float y[32];
-            uint8_t* code_dst = p.codes + row * (p.K >> 1) + (k0 >> 1);
             // ---- first MX block
             tmem_ld_32x32b_x32(taddr, raw);
             tmem_ld_wait();
-            if (MODE == kModeSR) sr_draws32(p.keys, p.stream_tag, i_next, n0);
+            if (MODE == kModeSR) sr_draws32(p.keys, tag_next, i_next, n0);
 #pragma unroll
             for (int i = 0; i < 32; ++i) y[i] = __uint_as_float(raw[i]) * cg;   // exact no-op unless g is 32 or 128
             if (MODE == kModeDump) {
                 if (live) {
-                    float4* dst = reinterpret_cast<float4*>(p.y_out + row * p.K + k0);
+                    float4* dst = reinterpret_cast<float4*>(y_dst);
 #pragma unroll
                     for (int i = 0; i < 8; ++i) dst[i] = make_float4(y[4 * i], y[4 * i + 1], y[4 * i + 2], y[4 * i + 3]);
                 }
@@ -244,12 +274,12 @@ quantize_tc_kernel(const __grid_constant__ CUtensorMap tmap_x, const QParams p) 
             tc_fence_before_sync();
             __syncwarp();
             if (lane == 0) mbar_arrive(&acc_empty[b]);
-            if (MODE == kModeSR) sr_draws32(p.keys, p.stream_tag, i_next + 32, n1);
+            if (MODE == kModeSR) sr_draws32(p.keys, tag_next, i_next + 32, n1);
 #pragma unroll
             for (int i = 0; i < 32; ++i) y[i] = __uint_as_float(raw[i]) * cg;
             if (MODE == kModeDump) {
                 if (live) {
-                    float4* dst = reinterpret_cast<float4*>(p.y_out + row * p.K + k0 + 32);
+                    float4* dst = reinterpret_cast<float4*>(y_dst + 32);
 #pragma unroll
                     for (int i = 0; i < 8; ++i) dst[i] = make_float4(y[4 * i], y[4 * i + 1], y[4 * i + 2], y[4 * i + 3]);
                 }
@@ -257,9 +287,7 @@ quantize_tc_kernel(const __grid_constant__ CUtensorMap tmap_x, const QParams p) 
                 quantize_block32_rw<MODE>(y, rw1, packed, sb1, p.pipe);
                 if (live) {
                     *reinterpret_cast<uint4*>(code_dst + 16) = make_uint4(packed[0], packed[1], packed[2], packed[3]);
-                    const int64_t so = p.sf_native ? ((int64_t)(rt * nkc + kt) * 512 + lane * 16 + q * 4 + half * 2)
-                                                   : row * nkb + (k0 >> 5);
-                    *reinterpret_cast<uint16_t*>(p.scales + so) = (uint16_t)(sb0 | (sb1 << 8));
+                    *reinterpret_cast<uint16_t*>(scale_dst) = (uint16_t)(sb0 | (sb1 << 8));
                 }
             }
             if (MODE == kModeSR) {
@@ -288,7 +316,7 @@ bool quant_tc_eligible(const QuantArgs& a) {
     const int64_t K = a.reduce_dim == 1 ? a.cols : a.rows;
     const int64_t R = a.reduce_dim == 1 ? a.rows : a.cols;
     const int64_t tiles = ((R + kTile - 1) / kTile) * (K / kTile);          // tile indices are 32-bit in the kernel
-    return (a.g == 32 || a.g == 64 || a.g == 128) && K % kTile == 0 && tiles < (int64_t(1) << 30) && a.has_tmap;
+    return (a.g == 32 || a.g == 64 || a.g == 128) && K % kTile == 0 && tiles < (int64_t(1) << 28) && a.has_tmap;
 }
 
 cudaError_t quant_tc_init() {
@@ -299,18 +327,32 @@ cudaError_t quant_tc_init() {
     return cudaFuncSetAttribute(quantize_tc_kernel<kModeDump>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kSmemQ);
 }
 
-cudaError_t launch_quantize_tc(const QuantArgs& a, bool dump_y, cudaStream_t stream) {
+// Quantise n (1..kQuantMaxViews) eligible operand views that share g, seed, rounding and scale layout in one launch.
+cudaError_t launch_quantize_tc_group(const QuantArgs* a, int n, bool dump_y, cudaStream_t stream) {
+    if (n < 1 || n > kQuantMaxViews) return cudaErrorInvalidValue;
     QParams p;
-    p.R = a.reduce_dim == 1 ? a.rows : a.cols;
-    p.K = a.reduce_dim == 1 ? a.cols : a.rows;
-    p.r_tiles = (p.R + kTile - 1) / kTile;
-    p.k_tiles = p.K / kTile;
-    p.reduce_dim = a.reduce_dim; p.g = a.g; p.rounding = a.rounding;
-    p.seed = a.seed; p.stream_tag = a.stream_tag;
-    p.codes = a.codes; p.scales = a.scales; p.sf_native = a.sf_native; p.y_out = a.y_out;
+    QMaps maps;
+    uint32_t tiles = 0;
+    for (int v = 0; v < n; ++v) {
+        QView& w = p.view[v];
+        w.R = a[v].reduce_dim == 1 ? a[v].rows : a[v].cols;
+        w.K = a[v].reduce_dim == 1 ? a[v].cols : a[v].rows;
+        w.r_tiles = (uint32_t)((w.R + kTile - 1) / kTile);
+        w.k_tiles = (uint32_t)(w.K / kTile);
+        w.tile_begin = tiles;
+        tiles += w.r_tiles * w.k_tiles;
+        w.reduce_dim = a[v].reduce_dim;
+        w.stream_tag = a[v].stream_tag;
+        w.codes = a[v].codes; w.scales = a[v].scales; w.y_out = a[v].y_out;
+        maps.x[v] = a[v].tmap_x;
+    }
+    for (int v = n; v < kQuantMaxViews; ++v) { p.view[v] = p.view[0]; p.view[v].tile_begin = 0xFFFFFFFFu; maps.x[v] = maps.x[0]; }
+    p.n_views = n;
+    p.n_tiles = tiles;
+    p.g = a[0].g; p.sf_native = a[0].sf_native; p.seed = a[0].seed;
     p.pipe = make_pipe_consts();
     {   // Philox key schedule: key_i = key_0 + i * (0x9E3779B9, 0xBB67AE85)
-        uint32_t k0 = (uint32_t)a.seed, k1 = (uint32_t)(a.seed >> 32);
+        uint32_t k0 = (uint32_t)p.seed, k1 = (uint32_t)(p.seed >> 32);
         for (int i = 0; i < 10; ++i) {
             p.keys.k0[i] = k0; p.keys.k1[i] = k1;
             k0 += 0x9E3779B9u; k1 += 0xBB67AE85u;
@@ -321,15 +363,18 @@ cudaError_t launch_quantize_tc(const QuantArgs& a, bool dump_y, cudaStream_t str
     if (e != cudaSuccess) return e;
     e = cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
     if (e != cudaSuccess) return e;
-    const int64_t tiles = p.r_tiles * p.k_tiles;
-    const unsigned grid = (unsigned)(tiles < sms ? tiles : sms);
+    const unsigned grid = tiles < (uint32_t)sms ? tiles : (unsigned)sms;
     if (dump_y)
-        quantize_tc_kernel<kModeDump><<<grid, kThreadsQ, kSmemQ, stream>>>(a.tmap_x, p);
-    else if (a.rounding == 0)
-        quantize_tc_kernel<kModeSR><<<grid, kThreadsQ, kSmemQ, stream>>>(a.tmap_x, p);
+        quantize_tc_kernel<kModeDump><<<grid, kThreadsQ, kSmemQ, stream>>>(maps, p);
+    else if (a[0].rounding == 0)
+        quantize_tc_kernel<kModeSR><<<grid, kThreadsQ, kSmemQ, stream>>>(maps, p);
     else
-        quantize_tc_kernel<kModeRN><<<grid, kThreadsQ, kSmemQ, stream>>>(a.tmap_x, p);
+        quantize_tc_kernel<kModeRN><<<grid, kThreadsQ, kSmemQ, stream>>>(maps, p);
     return cudaGetLastError();
+}
+
+cudaError_t launch_quantize_tc(const QuantArgs& a, bool dump_y, cudaStream_t stream) {
+    return launch_quantize_tc_group(&a, 1, dump_y, stream);
 }
 
 }  // namespace mx
