@@ -23,7 +23,7 @@ struct Runtime {
     std::once_flag once;
     mxfp4_status status = MXFP4_OK;
     EncodeTiledFn encode = nullptr;
-    bool gemm_pair = false;      // CTA-pair GEMM (gemm_pair.cu) only with MXFP4_GEMM_PAIR=1: measured slightly slower
+    bool gemm_pair = true;       // CTA-pair GEMM (gemm_pair.cu); MXFP4_GEMM_PAIR=0 selects the 1-CTA kernel (gemm.cu)
 };
 Runtime g_rt;
 
@@ -49,7 +49,7 @@ mxfp4_status runtime_init() {
         g_rt.encode = reinterpret_cast<EncodeTiledFn>(fn);
         if (mx::gemm_init() != cudaSuccess || mx::gemm_pair_init() != cudaSuccess || mx::quant_tc_init() != cudaSuccess) g_rt.status = MXFP4_ERR_CUDA;
         const char* pair = getenv("MXFP4_GEMM_PAIR");
-        g_rt.gemm_pair = pair != nullptr && pair[0] == '1';
+        g_rt.gemm_pair = !(pair != nullptr && pair[0] == '0');
     });
     return g_rt.status;
 }
@@ -106,6 +106,20 @@ void attach_input_map(QuantArgs& a) {
     a.has_tmap = r == CUDA_SUCCESS;
 }
 
+// Tensor map over the output C [M, N] for the pair kernel's stores: box = 64 bytes of a row x 32 rows, 64-byte swizzle.
+bool make_output_map(CUtensorMap* map, void* C, int64_t M, int64_t N, int64_t ldc, bool fp32) {
+    const int64_t es = fp32 ? 4 : 2;
+    if ((reinterpret_cast<uintptr_t>(C) & 15u) != 0 || (ldc * es) % 16 != 0 || M > 0x7FFFFFFF || N > 0x7FFFFFFF) return false;
+    const cuuint64_t dims[2] = {(cuuint64_t)N, (cuuint64_t)M};
+    const cuuint64_t strides[1] = {(cuuint64_t)(ldc * es)};
+    const cuuint32_t box[2] = {(cuuint32_t)(64 / es), 32};
+    const cuuint32_t elem_strides[2] = {1, 1};
+    const CUresult r = g_rt.encode(map, fp32 ? CU_TENSOR_MAP_DATA_TYPE_FLOAT32 : CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, C, dims, strides,
+                                   box, elem_strides, CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_64B,
+                                   CU_TENSOR_MAP_L2_PROMOTION_NONE, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+    return r == CUDA_SUCCESS;
+}
+
 mxfp4_status gemm_impl(const uint8_t* A_codes, const uint8_t* A_scales, const uint8_t* B_codes, const uint8_t* B_scales, int64_t M,
                        int64_t N, int64_t K, float alpha, void* C, int64_t ldc, int out_dtype, cudaStream_t stream) {
     GemmArgs a;
@@ -120,6 +134,7 @@ mxfp4_status gemm_impl(const uint8_t* A_codes, const uint8_t* A_scales, const ui
     if (a.use_pair) {
         st = make_codes_map(&a.tmap_b_half, B_codes, N, K, 128);
         if (st != MXFP4_OK) return st;
+        a.has_tmap_c = make_output_map(&a.tmap_c, C, M, N, ldc, a.out_fp32 != 0);
         return mx::launch_gemm_pair(a, stream) == cudaSuccess ? MXFP4_OK : MXFP4_ERR_CUDA;
     }
     return mx::launch_gemm(a, stream) == cudaSuccess ? MXFP4_OK : MXFP4_ERR_CUDA;

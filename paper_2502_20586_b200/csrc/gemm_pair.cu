@@ -33,10 +33,15 @@ constexpr uint32_t kStageB = 2 * kAB;                       // 32 KB: A rows + B
 constexpr int kSfSlotsP = kStagesP;                         // scale ring: shared-memory slot i feeds TMEM slot i; same ring
                                                             // index as the operand stages so ONE commit frees both
 constexpr uint32_t kSfSlotB = kSfaB + kSfbB;                // 3 KB
-constexpr uint32_t kSmemP = kStagesP * kStageB + kSfSlotsP * kSfSlotB + 1024 + 512;
+constexpr uint32_t kEpiBuf = 2048;                          // epilogue staging: 32 rows x 64 B, two buffers per epilogue warp
+constexpr uint32_t kEpiB = 4 * 2 * kEpiBuf;
+constexpr uint32_t kBarB = 256;
+// The dynamic shared-memory window is at least 256-byte aligned, so rounding its base up to 1024 costs at most 768 bytes.
+constexpr uint32_t kSmemP = kStagesP * kStageB + kSfSlotsP * kSfSlotB + kEpiB + kBarB + 768;
+static_assert(kSmemP <= 232448, "over the 227 KB shared-memory limit");
 constexpr uint32_t kAccColP = 0, kSfColP = 256, kSfSlotColsP = 24;
 constexpr int kGroupMP = 8;                                 // rasterisation: 8 pair-tiles (2048 rows) share B tiles in L2
-constexpr int kThreadsP = 11 * 32;
+constexpr int kThreadsP = 12 * 32;
 
 struct ParamsP {
     const uint8_t* sfa;
@@ -46,6 +51,7 @@ struct ParamsP {
     float alpha;
     int out_fp32;
     int m_tiles, n_tiles;                                   // in pair tiles
+    int c_tma;                                              // C goes out through tmap_c (else plain stores)
 };
 
 __device__ __forceinline__ void tile_coords_p(int t, int m_tiles, int n_tiles, int& mt, int& nt) {
@@ -59,17 +65,20 @@ __device__ __forceinline__ void tile_coords_p(int t, int m_tiles, int n_tiles, i
 }
 
 __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(kThreadsP, 1)
-gemm_mxf4_pair_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant__ CUtensorMap tmap_b, const ParamsP p) {
+gemm_mxf4_pair_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant__ CUtensorMap tmap_b,
+                      const __grid_constant__ CUtensorMap tmap_c, const ParamsP p) {
     extern __shared__ uint8_t smem_raw[];
     uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
     uint8_t* sf_ring = smem + kStagesP * kStageB;
-    uint64_t* bars = reinterpret_cast<uint64_t*>(sf_ring + kSfSlotsP * kSfSlotB);
-    uint64_t* full_bar = bars;                              // [kStagesP] leader: A and B halves of both CTAs landed
-    uint64_t* empty_bar = full_bar + kStagesP;              // [kStagesP] per CTA: stage free (pair commit)
+    uint8_t* epi_ring = sf_ring + kSfSlotsP * kSfSlotB;
+    uint64_t* bars = reinterpret_cast<uint64_t*>(epi_ring + kEpiB);
+    uint64_t* full_bar = bars;                              // [kStagesP] leader: operands of both CTAs landed AND their
+                                                            //            scales are in TMEM (1 expect_tx arrival + 8 movers)
+    uint64_t* empty_bar = full_bar + kStagesP;              // [kStagesP] per CTA: stage and scale slot free (pair commit)
     uint64_t* sfl_full = empty_bar + kStagesP;              // [kSfSlotsP] per CTA: scale tiles landed in the ring slot
-    uint64_t* sf_full = sfl_full + kSfSlotsP;                // [kSfSlotsP] leader: scales of both CTAs are in TMEM
-    uint64_t* sf_empty = sf_full + kSfSlotsP;               // [kSfSlotsP] per CTA: scale slot free (pair commit)
-    uint64_t* tmem_full = sf_empty + kSfSlotsP;             // per CTA: accumulator complete (pair commit)
+    uint64_t* sfl_empty = sfl_full + kSfSlotsP;             // [kSfSlotsP] per CTA: the movers have read the ring slot (4 arrivals)
+    uint64_t* turn = sfl_empty + kSfSlotsP;                 // [2] leader: baton between the two MMA issuers
+    uint64_t* tmem_full = turn + 2;                         // per CTA: accumulator complete (pair commit)
     uint64_t* tmem_empty = tmem_full + 1;                   // leader: both CTAs drained their accumulators
     uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(tmem_empty + 1);
     volatile uint32_t* abort_flag = tmem_slot + 1;
@@ -84,14 +93,16 @@ gemm_mxf4_pair_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_c
     const uint32_t total = my_tiles * (uint32_t)num_kt;
 
     if (threadIdx.x == 0) {
-        for (int s = 0; s < kStagesP; ++s) { mbar_init(&full_bar[s], 1); mbar_init(&empty_bar[s], 1); }
-        for (int s = 0; s < kSfSlotsP; ++s) { mbar_init(&sfl_full[s], 1); mbar_init(&sf_full[s], 8); mbar_init(&sf_empty[s], 1); }
+        for (int s = 0; s < kStagesP; ++s) { mbar_init(&full_bar[s], 1 + 8); mbar_init(&empty_bar[s], 1); }
+        for (int s = 0; s < kSfSlotsP; ++s) { mbar_init(&sfl_full[s], 1); mbar_init(&sfl_empty[s], 4); }
+        mbar_init(&turn[0], 1); mbar_init(&turn[1], 1);
         mbar_init(tmem_full, 1);
         mbar_init(tmem_empty, 8);
         *abort_flag = 0;
         mbar_fence_init();
         prefetch_tensormap(&tmap_a);
         prefetch_tensormap(&tmap_b);
+        if (p.c_tma) prefetch_tensormap(&tmap_c);
     }
     if (warp == 1) {
         tmem_alloc_pair(tmem_slot, 512);
@@ -123,36 +134,52 @@ gemm_mxf4_pair_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_c
             }
             if (!ok) *abort_flag = 1;
         }
-    } else if (warp == 1) {
-        // ------------------------------------------------------------------ MMA issuer (leader CTA only)
-        if (lane == 0 && rank == 0) {
+    } else if (warp == 1 || warp == 11) {
+        // ------------------------------------------------------------------ MMA issuers (leader CTA only)
+        // Issuing one pair MMA occupies its thread for ~90 cycles and a commit for ~100, which is more than the
+        // tensor pipe needs for the four MMAs of a step.  Two threads therefore take the steps in turn (even steps
+        // warp 1, odd steps warp 11): while one issues, the other has already waited for its operands and then
+        // commits.  A baton (mbarrier turn[]) keeps the MMAs in step order, so accumulation order is fixed.
+        if (rank == 0 && lane == 0) {
             // instruction descriptor: A, B = E2M1 (1), scale = UE8M0 (1), K-major, N >> 3 at bit 17, M >> 4 at bit 24
-            const uint32_t idesc_base = (1u << 7) | (1u << 10) | ((uint32_t)(PN >> 3) << 17) | (1u << 23) | ((uint32_t)(PM >> 4) << 24);
-            uint32_t tile_i = 0;
+            const uint32_t idesc0 = (1u << 7) | (1u << 10) | ((uint32_t)(PN >> 3) << 17) | (1u << 23) | ((uint32_t)(PM >> 4) << 24);
+            const uint32_t idesc1 = idesc0 | (2u << 29) | (2u << 4);          // scale bytes 2, 3 of the 32-bit column
+            const uint64_t desc0 = make_smem_desc(smem_u32(smem), 16, 1024, 2);
+            const uint32_t desc_hi = (uint32_t)(desc0 >> 32);
+            const uint32_t a_lo0 = (uint32_t)desc0;
+            const bool k_tail = (nkc & 1) != 0;                               // last step holds 128 elements only
+            const uint32_t acc = tmem_base + kAccColP;
+            const uint32_t me = warp == 1 ? 0u : 1u;
+            uint32_t s = me % kStagesP, ph = 0, tile_i = 0, n = 0;
+            int kt = (int)me;
+            while (kt >= num_kt) { kt -= num_kt; ++tile_i; }
             bool ok = true;
-            for (uint32_t it = 0; it < total; ++it) {
-                const int kt = (int)(it % (uint32_t)num_kt);
-                const int s = it % kStagesP, slot = it % kSfSlotsP;
+            for (uint32_t it = me; it < total; it += 2, ++n) {
                 if (kt == 0) {
                     if (!(ok = mbar_wait(tmem_empty, (tile_i & 1) ^ 1, abort_flag))) break;
                 }
-                if (!(ok = mbar_wait(&full_bar[s], (it / kStagesP) & 1, abort_flag))) break;
-                if (!(ok = mbar_wait(&sf_full[slot], (it / kSfSlotsP) & 1, abort_flag))) break;
+                if (!(ok = mbar_wait(&full_bar[s], ph, abort_flag))) break;
+                if (!(ok = mbar_wait_spin(&turn[me], (n & 1) ^ me ^ 1, abort_flag))) break;   // the step before mine is issued
                 tc_fence_after_sync();
-                const uint32_t st = smem_u32(smem + s * kStageB);
-                const int nch = min(2, nkc - 2 * kt);
-                const uint32_t sfa_t = tmem_base + kSfColP + slot * kSfSlotColsP, sfb_t = sfa_t + 8;
-                for (int kb = 0; kb < 2 * nch; ++kb) {
-                    const uint64_t adesc = make_smem_desc(st + kb * 32, 16, 1024, 2);
-                    const uint64_t bdesc = make_smem_desc(st + kAB + kb * 32, 16, 1024, 2);
-                    const uint32_t sf_id = (uint32_t)(kb & 1) * 2u;
-                    const uint32_t idesc = idesc_base | (sf_id << 29) | (sf_id << 4);
-                    tc_mma_mxf4_pair(tmem_base + kAccColP, adesc, bdesc, idesc,
-                                     (sfa_t + 4 * (kb >> 1)) | (sf_id << 30), (sfb_t + 8 * (kb >> 1)) | (sf_id << 30),
-                                     (kt | kb) != 0 ? 1u : 0u);
+                const uint32_t a_lo = a_lo0 + s * (kStageB >> 4), b_lo = a_lo + (kAB >> 4);
+                const uint32_t sfa_t = tmem_base + kSfColP + s * kSfSlotColsP, sfb_t = sfa_t + 8;
+                const uint32_t hi2 = 2u << 30;
+                const bool last = kt == num_kt - 1;
+                auto D = [&](uint32_t lo) { return ((uint64_t)desc_hi << 32) | lo; };
+                tc_mma_mxf4_pair(acc, D(a_lo), D(b_lo), idesc0, sfa_t, sfb_t, kt != 0 ? 1u : 0u);
+                tc_mma_mxf4_pair(acc, D(a_lo + 2), D(b_lo + 2), idesc1, sfa_t | hi2, sfb_t | hi2, 1u);
+                if (!(last && k_tail)) {
+                    tc_mma_mxf4_pair(acc, D(a_lo + 4), D(b_lo + 4), idesc0, sfa_t + 4, sfb_t + 8, 1u);
+                    tc_mma_mxf4_pair(acc, D(a_lo + 6), D(b_lo + 6), idesc1, (sfa_t + 4) | hi2, (sfb_t + 8) | hi2, 1u);
                 }
+                tc_fence_before_sync();
+                mbar_arrive(&turn[me ^ 1]);                                    // pass the baton
                 tc_commit_pair(&empty_bar[s]);                                 // frees the operand stage and the scale slot
-                if (kt == num_kt - 1) { tc_commit_pair(tmem_full); ++tile_i; }
+                if (last) tc_commit_pair(tmem_full);
+                s += 2;
+                if (s >= (uint32_t)kStagesP) { s -= kStagesP; ph ^= 1; }
+                kt += 2;
+                while (kt >= num_kt) { kt -= num_kt; ++tile_i; }
             }
             if (!ok) *abort_flag = 1;
         }
@@ -169,8 +196,8 @@ gemm_mxf4_pair_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_c
                 const int n_row_tiles = min(2, (int)((p.N - (int64_t)nt * PN + 127) >> 7));
                 for (int kt = 0; kt < num_kt; ++kt, ++it) {
                     const int slot = it % kSfSlotsP;
-                    // the slot's previous scales (shared memory and TMEM) are dead once the MMAs that read them completed
-                    if (!(ok = mbar_wait(&empty_bar[slot], ((it / kSfSlotsP) & 1) ^ 1, abort_flag))) break;
+                    // the ring slot is free once the movers have carried its previous contents to TMEM
+                    if (!(ok = mbar_wait(&sfl_empty[slot], ((it / kSfSlotsP) & 1) ^ 1, abort_flag))) break;
                     uint8_t* dst = sf_ring + slot * kSfSlotB;
                     const int nch = min(2, nkc - 2 * kt);
                     mbar_expect_tx(&sfl_full[slot], (uint32_t)nch * kSfTile * ((has_a ? 1u : 0u) + (uint32_t)n_row_tiles));
@@ -189,7 +216,11 @@ gemm_mxf4_pair_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_c
         bool ok = true;
         for (uint32_t it = 0; it < total; ++it) {
             const int slot = it % kSfSlotsP;
-            if (lane == 0) ok = mbar_wait(&sfl_full[slot], (it / kSfSlotsP) & 1, abort_flag);
+            if (lane == 0) {
+                // scales landed in shared memory, and the MMAs that read this TMEM slot's previous scales are done
+                ok = mbar_wait(&sfl_full[slot], (it / kSfSlotsP) & 1, abort_flag) &&
+                     mbar_wait(&empty_bar[slot], ((it / kSfSlotsP) & 1) ^ 1, abort_flag);
+            }
             ok = __shfl_sync(0xffffffffu, ok, 0);
             if (!ok) break;
             tc_fence_after_sync();
@@ -200,13 +231,37 @@ gemm_mxf4_pair_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_c
             tmem_st_wait();
             tc_fence_before_sync();
             __syncwarp();
-            if (lane == 0) mbar_arrive_cluster(&sf_full[slot], 0);
+            if (lane == 0) { mbar_arrive(&sfl_empty[slot]); mbar_arrive_cluster(&full_bar[slot], 0); }
         }
         if (!ok && lane == 0) *abort_flag = 1;
     } else {
         // ------------------------------------------------------------------ epilogue (both CTAs, own 128 rows)
+        // TMEM -> registers -> (alpha, convert) -> shared memory -> TMA store.  Each warp owns the 32 accumulator
+        // lanes of its quadrant and two 2 KB staging buffers (32 rows x 64 bytes, 64-byte swizzle, so the row-per-lane
+        // writes are conflict-free); the accumulator is handed back as soon as its last column is in registers.
         const int q = warp & 3;
+        uint8_t* stage0 = epi_ring + q * 2 * kEpiBuf;
+        uint32_t n_stores = 0;                                  // bulk groups this warp committed so far
         bool ok = true;
+        // One staged block: 16 registers = 64 bytes of this lane's row, columns [col, col + 64 B).
+        auto put = [&](const uint32_t (&w)[16], int32_t col, int32_t row0, bool in_range) {
+            uint8_t* buf = stage0 + (n_stores & 1) * kEpiBuf;
+            if (n_stores >= 2) {                                // the store that last read this buffer must be done with it
+                if (lane == 0) bulk_wait_group_read<1>();
+                __syncwarp();
+            }
+            uint4* dst = reinterpret_cast<uint4*>(buf + lane * 64);
+            const int sw = (lane >> 1) & 3;
+#pragma unroll
+            for (int j = 0; j < 4; ++j) dst[j ^ sw] = make_uint4(w[4 * j], w[4 * j + 1], w[4 * j + 2], w[4 * j + 3]);
+            fence_proxy_async_smem();
+            __syncwarp();
+            if (lane == 0) {
+                if (in_range) tma_store_2d(&tmap_c, buf, col, row0);
+                bulk_commit_group();
+            }
+            ++n_stores;
+        };
         for (uint32_t tl = 0; tl < my_tiles; ++tl) {
             int mt, nt;
             tile_coords_p((int)(pair + tl * num_pairs), p.m_tiles, p.n_tiles, mt, nt);
@@ -214,15 +269,70 @@ gemm_mxf4_pair_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_c
             ok = __shfl_sync(0xffffffffu, ok, 0);
             if (!ok) break;
             tc_fence_after_sync();
-            const int64_t row = (int64_t)mt * PM + (int64_t)rank * 128 + q * 32 + lane;
+            const int64_t row0 = (int64_t)mt * PM + (int64_t)rank * 128 + q * 32;
+            const int64_t row = row0 + lane;
             const int64_t col0 = (int64_t)nt * PN;
+            int n_chunks = PN / 32;
+            if (p.c_tma && !p.out_fp32) {
+                // bf16: drain the whole accumulator into registers first (packed pairs), hand it back, then store.
+                uint32_t out[PN / 2];
+#pragma unroll
+                for (int c = 0; c < PN / 32; ++c) {
+                    uint32_t r[32];
+                    tmem_ld_32x32b_x32(tmem_base + kAccColP + ((uint32_t)(q * 32) << 16) + c * 32, r);
+                    tmem_ld_wait();
+#pragma unroll
+                    for (int j = 0; j < 16; ++j) {
+                        const __nv_bfloat162 h = __floats2bfloat162_rn(__uint_as_float(r[2 * j]) * p.alpha,
+                                                                       __uint_as_float(r[2 * j + 1]) * p.alpha);
+                        out[16 * c + j] = *reinterpret_cast<const uint32_t*>(&h);
+                    }
+                }
+                tc_fence_before_sync();
+                __syncwarp();
+                if (lane == 0) mbar_arrive_cluster(tmem_empty, 0);
+#pragma unroll
+                for (int c = 0; c < PN / 32; ++c) {
+                    uint32_t w[16];
+#pragma unroll
+                    for (int j = 0; j < 16; ++j) w[j] = out[16 * c + j];
+                    const int64_t col = col0 + c * 32;
+                    put(w, (int32_t)col, (int32_t)row0, row0 < p.M && col < p.N);
+                }
+                n_chunks = 0;
+            }
 #pragma unroll 1
-            for (int c = 0; c < PN / 32; ++c) {
+            for (int c = 0; c < n_chunks; ++c) {
                 uint32_t r[32];
                 tmem_ld_32x32b_x32(tmem_base + kAccColP + ((uint32_t)(q * 32) << 16) + c * 32, r);
                 tmem_ld_wait();
+                if (c == n_chunks - 1) {                        // accumulator drained: the next tile's MMAs may start
+                    tc_fence_before_sync();
+                    __syncwarp();
+                    if (lane == 0) mbar_arrive_cluster(tmem_empty, 0);
+                }
                 const int64_t col = col0 + c * 32;
-                if (row < p.M && col < p.N) {
+                if (p.c_tma) {
+                    const bool in_range = row0 < p.M && col < p.N;
+                    if (p.out_fp32) {
+                        uint32_t w[16];
+#pragma unroll
+                        for (int h = 0; h < 2; ++h) {
+#pragma unroll
+                            for (int j = 0; j < 16; ++j) w[j] = __float_as_uint(__uint_as_float(r[16 * h + j]) * p.alpha);
+                            put(w, (int32_t)col + 16 * h, (int32_t)row0, in_range && col + 16 * h < p.N);
+                        }
+                    } else {
+                        uint32_t w[16];
+#pragma unroll
+                        for (int j = 0; j < 16; ++j) {
+                            const __nv_bfloat162 h = __floats2bfloat162_rn(__uint_as_float(r[2 * j]) * p.alpha,
+                                                                           __uint_as_float(r[2 * j + 1]) * p.alpha);
+                            w[j] = *reinterpret_cast<const uint32_t*>(&h);
+                        }
+                        put(w, (int32_t)col, (int32_t)row0, in_range);
+                    }
+                    } else if (row < p.M && col < p.N) {
                     const int nvalid = (int)min((int64_t)32, p.N - col);      // multiple of 8
                     if (p.out_fp32) {
                         float* dst = static_cast<float*>(p.C) + row * p.ldc + col;
@@ -249,10 +359,8 @@ gemm_mxf4_pair_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_c
                     }
                 }
             }
-            tc_fence_before_sync();
-            __syncwarp();
-            if (lane == 0) mbar_arrive_cluster(tmem_empty, 0);
         }
+        if (lane == 0) bulk_wait_group<0>();                         // every store has left shared memory and is visible
         if (!ok && lane == 0) *abort_flag = 1;
     }
 
@@ -289,7 +397,8 @@ cudaError_t launch_gemm_pair(const GemmArgs& a, cudaStream_t stream) {
     if (e != cudaSuccess) return e;
     const int tiles = p.m_tiles * p.n_tiles;
     const int pairs = tiles < sms / 2 ? tiles : sms / 2;
-    gemm_mxf4_pair_kernel<<<2 * pairs, kThreadsP, kSmemP, stream>>>(a.tmap_a, a.tmap_b_half, p);
+    p.c_tma = a.has_tmap_c ? 1 : 0;
+    gemm_mxf4_pair_kernel<<<2 * pairs, kThreadsP, kSmemP, stream>>>(a.tmap_a, a.tmap_b_half, a.tmap_c, p);
     return cudaGetLastError();
 }
 

@@ -37,6 +37,8 @@ struct GemmArgs {
     CUtensorMap tmap_a;   // codes [M, K/2] bytes, box 128 B x 128 rows, 128-byte swizzle
     CUtensorMap tmap_b;   // codes [N, K/2] bytes, box 128 B x BN rows
     CUtensorMap tmap_b_half;   // same tensor, box 128 B x 128 rows (CTA-pair kernel: each CTA loads half a B tile)
+    CUtensorMap tmap_c;   // output [M, N] (leading dimension ldc): box 64 bytes x 32 rows, 64-byte swizzle (pair kernel's stores)
+    bool has_tmap_c;      // false when C cannot be described by a tensor map: the kernel then stores directly
     bool use_pair;        // run the CTA-pair kernel (gemm_pair.cu)
     const uint8_t* sfa;   // native scale layout
     const uint8_t* sfb;

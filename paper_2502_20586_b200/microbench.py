@@ -29,6 +29,7 @@ def _time(fn, iters, flush_buf):
         if flush_buf is not None:
             _flush_l2(flush_buf)
         a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        torch.cuda._sleep(400000)        # keep the GPU busy while the host enqueues, so host latency is not timed
         a.record(); fn(); b.record()
         torch.cuda.synchronize()
         times.append(a.elapsed_time(b))
