@@ -116,6 +116,11 @@ MXFP4_API size_t mxfp4_linear_backward_workspace(int64_t b, int64_t m, int64_t n
  *   vector; dX = alpha Q1 Q2^T, dW = alpha Q3 Q4^T with alpha = 16/9 iff rounding = SR.
  *   workspace: device scratch of at least mxfp4_linear_backward_workspace() bytes, 256-byte aligned;
  *   its contents are overwritten.  Calls sharing a workspace must be stream-ordered.
+ *   Ordering: everything the call does is ordered after prior work of `cuda_stream` and before later work of it.
+ *   For large shapes the two GEMMs (independent of each other) run side by side: the call forks onto a
+ *   library-owned side stream after the quantisers and joins back into `cuda_stream` before it returns (event
+ *   record / wait only, no host synchronisation).  The side stream and its two events are created once per host
+ *   thread at the first such call; MXFP4_FORK_JOIN=0 in the environment keeps every launch on `cuda_stream`.
  */
 MXFP4_API mxfp4_status mxfp4_linear_backward(const void* dY, const void* X, const void* W,
                                    int64_t b, int64_t m, int64_t n, int g, int rounding, uint64_t seed,

@@ -54,6 +54,33 @@ mxfp4_status runtime_init() {
     return g_rt.status;
 }
 
+// Side stream and events for running the two independent GEMMs of a backward call side by side (fork / join around
+// the caller's stream): the second GEMM's CTAs move onto SMs as the first one's last wave drains.  One set per host
+// thread, created at its first large call and kept; on any failure the call simply stays on the caller's stream.
+struct ForkJoin {
+    bool tried = false, ok = false;
+    int device = -1;
+    cudaStream_t side = nullptr;
+    cudaEvent_t fork = nullptr, join = nullptr;
+};
+ForkJoin* fork_join() {
+    static thread_local ForkJoin fj;
+    int dev = -1;
+    if (cudaGetDevice(&dev) != cudaSuccess) return nullptr;
+    if (!fj.tried) {
+        fj.tried = true;
+        fj.device = dev;
+        int lo = 0, hi = 0;
+        fj.ok = cudaDeviceGetStreamPriorityRange(&lo, &hi) == cudaSuccess &&
+                cudaStreamCreateWithPriority(&fj.side, cudaStreamNonBlocking, lo) == cudaSuccess &&
+                cudaEventCreateWithFlags(&fj.fork, cudaEventDisableTiming) == cudaSuccess &&
+                cudaEventCreateWithFlags(&fj.join, cudaEventDisableTiming) == cudaSuccess;
+        const char* e = getenv("MXFP4_FORK_JOIN");
+        if (e != nullptr && e[0] == '0') fj.ok = false;
+    }
+    return fj.ok && fj.device == dev ? &fj : nullptr;
+}
+
 bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
 bool valid_g(int g) { return g == 0 || g == 32 || g == 64 || g == 128 || g == 256; }
 int64_t round_up(int64_t v, int64_t a) { return (v + a - 1) / a * a; }
@@ -265,9 +292,18 @@ mxfp4_status mxfp4_linear_backward(const void* dY, const void* X, const void* W,
     }
     // lines 7-11: two MXFP4 GEMMs; the 16/9 un-does the two 3/4 pre-scales of Algorithm 2.
     const float alpha = rounding == MXFP4_ROUND_SR ? 16.0f / 9.0f : 1.0f;
+    // Large problems (never the ones the fixed-scratch variant accepts) run the two GEMMs fork / join.
+    const int64_t waves_dx = ((b + 255) / 256) * ((n + 255) / 256), waves_dw = ((m + 255) / 256) * ((n + 255) / 256);
+    ForkJoin* fj = ws.total > (size_t)MXFP4_STATIC_WORKSPACE_BYTES && waves_dx >= 74 && waves_dw >= 74 ? fork_join() : nullptr;
+    if (fj != nullptr && (cudaEventRecord(fj->fork, stream) != cudaSuccess || cudaStreamWaitEvent(fj->side, fj->fork, 0) != cudaSuccess))
+        return MXFP4_ERR_CUDA;
     st = gemm_impl(c[0], s[0], c[1], s[1], b, n, m, alpha, dX, n, out_dtype, stream);
     if (st != MXFP4_OK) return st;
-    return gemm_impl(c[2], s[2], c[3], s[3], m, n, b, alpha, dW, n, out_dtype, stream);
+    st = gemm_impl(c[2], s[2], c[3], s[3], m, n, b, alpha, dW, n, out_dtype, fj != nullptr ? fj->side : stream);
+    if (st != MXFP4_OK) return st;
+    if (fj != nullptr && (cudaEventRecord(fj->join, fj->side) != cudaSuccess || cudaStreamWaitEvent(stream, fj->join, 0) != cudaSuccess))
+        return MXFP4_ERR_CUDA;
+    return MXFP4_OK;
 }
 
 mxfp4_status mxfp4_device_status(void* cuda_stream) {
