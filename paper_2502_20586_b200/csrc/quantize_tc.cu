@@ -17,8 +17,8 @@
 //
 //   warp 0        TMA producer (two 64-column x 128-row boxes per tile, 128-byte swizzle, 4-stage ring)
 //   warp 1        MMA issuer (8 K=16 MMAs per tile into one of four 128-column TMEM accumulators)
-//   warps 2..17   epilogue, two groups of eight warps on alternate tiles: warp = (TMEM lane quadrant, 64 columns):
-//                 tcgen05.ld 32 columns at a time, release the accumulator, then scale / SR / pack / store
+//   warps 2..17   epilogue, four groups of four warps on alternate tiles: warp = TMEM lane quadrant, a thread owns one
+//                 output row of the tile: tcgen05.ld 32 columns at a time, scale / SR / pack / store per MX block
 // Every mbarrier wait is bounded; on expiry the CTA records a status word and unwinds.
 #include <cuda_bf16.h>
 
@@ -36,13 +36,17 @@ constexpr uint32_t kTileBytes = 2 * kBoxBytes;      // 32 KB
 constexpr uint32_t kTBytes = 2 * kBoxBytes;         // transform matrix, 128 x 128 bf16
 constexpr uint32_t kSmemQ = kStagesQ * kTileBytes + kTBytes + 1024 + 256;
 constexpr int kAccBufs = 4;                         // 4 x 128 TMEM columns
-constexpr int kEpiWarps = 16;
+constexpr int kEpiGroups = 4;                       // epilogue warp groups (one warp per TMEM lane quadrant), on alternate tiles
+constexpr int kEpiWarps = 4 * kEpiGroups;
 constexpr int kThreadsQ = (2 + kEpiWarps) * 32;
 
 struct QView {                 // one operand view: output operand [R, K] read from x [rows, cols]
     int64_t R, K;
     uint32_t r_tiles, k_tiles;
     uint32_t tile_begin;       // first index of this view in the launch's tile list
+    uint32_t n_tiles;          // r_tiles * k_tiles
+    uint32_t minor_count;      // tiles along the fast direction of the view's tile order (see locate_tile)
+    uint32_t d_major, d_minor; // an epilogue group's stride through the tile list, split by minor_count
     int reduce_dim;            // 1: K runs along x columns (x tile is the K-major operand); 0: along x rows (MN-major)
     uint32_t stream_tag;
     uint8_t* codes;
@@ -79,6 +83,7 @@ __device__ __forceinline__ uint32_t transform_entry(int n, int k, int g, const u
 struct TilePos {
     int v;
     uint32_t rt, kt;
+    uint32_t local;            // index inside the view
 };
 __device__ __forceinline__ TilePos locate_tile(const QParams& p, uint32_t t) {
     int v = 0;
@@ -88,8 +93,21 @@ __device__ __forceinline__ TilePos locate_tile(const QParams& p, uint32_t t) {
     const uint32_t local = t - p.view[v].tile_begin;
     TilePos pos;
     pos.v = v;
+    pos.local = local;
     if (p.view[v].reduce_dim == 1) { pos.rt = local / p.view[v].k_tiles; pos.kt = local - pos.rt * p.view[v].k_tiles; }
     else { pos.kt = local / p.view[v].r_tiles; pos.rt = local - pos.kt * p.view[v].r_tiles; }
+    return pos;
+}
+// The position `stride` tiles further on (stride = the view's d_major * minor_count + d_minor): additions only while
+// the walk stays inside the view.
+__device__ __forceinline__ TilePos advance_tile(const QParams& p, const TilePos& cur, uint32_t t_next) {
+    const QView& vw = p.view[cur.v];
+    TilePos pos = cur;
+    pos.local = cur.local + vw.d_major * vw.minor_count + vw.d_minor;
+    if (pos.local >= vw.n_tiles) return locate_tile(p, t_next);
+    uint32_t major = (vw.reduce_dim == 1 ? cur.rt : cur.kt) + vw.d_major, minor = (vw.reduce_dim == 1 ? cur.kt : cur.rt) + vw.d_minor;
+    if (minor >= vw.minor_count) { minor -= vw.minor_count; ++major; }
+    if (vw.reduce_dim == 1) { pos.rt = major; pos.kt = minor; } else { pos.kt = major; pos.rt = minor; }
     return pos;
 }
 
@@ -114,7 +132,7 @@ quantize_tc_kernel(const __grid_constant__ QMaps maps, const __grid_constant__ Q
 
     if (threadIdx.x == 0) {
         for (int s = 0; s < kStagesQ; ++s) { mbar_init(&full_bar[s], 1); mbar_init(&empty_bar[s], 1); }
-        for (int b = 0; b < kAccBufs; ++b) { mbar_init(&acc_full[b], 1); mbar_init(&acc_empty[b], kEpiWarps / 2); }
+        for (int b = 0; b < kAccBufs; ++b) { mbar_init(&acc_full[b], 1); mbar_init(&acc_empty[b], 4); }
         *abort_flag = 0;
         mbar_fence_init();
         for (int v = 0; v < p.n_views; ++v) prefetch_tensormap(&maps.x[v]);
@@ -201,99 +219,86 @@ quantize_tc_kernel(const __grid_constant__ QMaps maps, const __grid_constant__ Q
         }
     } else {
         // ------------------------------------------------------------------ epilogue
-        // Two groups of eight warps take alternate tiles (so one group's integer-heavy packing overlaps the other's
-        // multiply-heavy Philox rounds); inside a group a warp owns one TMEM lane quadrant and 64 of the 128 columns,
-        // i.e. two MX blocks per thread and tile.  The SR draws of the NEXT tile are computed while the current one
-        // is rounded: they depend only on element indices.
+        // Four groups of four warps take alternate tiles; inside a group a warp owns one TMEM lane quadrant, i.e. a
+        // thread owns one output row of the tile: four MX blocks, 64 bytes of codes, 4 scale bytes.  The SR draws of a
+        // block are computed while the block before it is rounded (for a tile's first block: at the end of the tile
+        // before); they depend only on element indices.
         const int e = warp - 2;
         const int q = warp & 3;                      // TMEM lane quadrant this warp may read
-        const int grp = e >> 3;
-        const int half = (e >> 2) & 1;
+        const int grp = e >> 2;
         const float cg = p.g == 32 ? 0.17677669529663687f : p.g == 128 ? 0.08838834764831845f : 1.0f;
-        const uint32_t stride = 2u * gridDim.x;
+        const uint32_t stride = (uint32_t)kEpiGroups * gridDim.x;
         const uint32_t lane_row = (uint32_t)(q * 32 + lane);
         bool ok = true;
 
         auto first_elem = [&](const TilePos& pos) -> uint64_t {          // linear index of this thread's first element
-            return (uint64_t)(pos.rt * (uint32_t)kTile + lane_row) * (uint64_t)p.view[pos.v].K +
-                   (uint64_t)(pos.kt * (uint32_t)kTile + (uint32_t)half * 64u);
+            return (uint64_t)(pos.rt * (uint32_t)kTile + lane_row) * (uint64_t)p.view[pos.v].K + (uint64_t)(pos.kt * (uint32_t)kTile);
         };
 
         uint32_t it = (uint32_t)grp;
         uint32_t t = blockIdx.x + it * gridDim.x;
         TilePos pos = locate_tile(p, t < num_tiles ? t : 0u);
-        uint32_t rw0[8], rw1[8];
-        if (MODE == kModeSR) {
-            const uint64_t i0 = first_elem(pos);
-            sr_draws32(p.keys, p.view[pos.v].stream_tag, i0, rw0);
-            sr_draws32(p.keys, p.view[pos.v].stream_tag, i0 + 32, rw1);
-        }
-        for (; t < num_tiles; t += stride, it += 2) {
+        uint32_t rw[8];
+        if (MODE == kModeSR) sr_draws32(p.keys, p.view[pos.v].stream_tag, first_elem(pos), rw);
+        for (; t < num_tiles; t += stride, it += kEpiGroups) {
             const int b = it % kAccBufs;
             const QView& vw = p.view[pos.v];
             const uint32_t rt = pos.rt, kt = pos.kt;
             const int64_t K = vw.K;
             const int64_t row = (int64_t)rt * kTile + lane_row;                 // output row
-            const int64_t k0 = (int64_t)kt * kTile + half * 64;
+            const int64_t k0 = (int64_t)kt * kTile;
             const bool live = row < vw.R;
             uint8_t* code_dst = vw.codes + row * (K >> 1) + (k0 >> 1);
             const uint32_t nkb = (uint32_t)(K >> 5), nkc = (nkb + 3) >> 2;
-            uint8_t* scale_dst = vw.scales + (p.sf_native ? ((int64_t)(rt * nkc + kt) * 512 + lane * 16 + q * 4 + half * 2)
-                                                           : row * nkb + (k0 >> 5));
+            uint8_t* scale_dst = vw.scales + (p.sf_native ? ((int64_t)(rt * nkc + kt) * 512 + lane * 16 + q * 4) : row * nkb + (k0 >> 5));
             float* y_dst = MODE == kModeDump ? vw.y_out + row * K + k0 : nullptr;
-            // position and draws of the next tile of this group (past the end: computed but not used)
-            pos = locate_tile(p, t + stride < num_tiles ? t + stride : 0u);
+            const uint64_t i_cur = first_elem(pos);
+            const uint32_t tag_cur = vw.stream_tag;
+            // position of the next tile of this group (past the end: computed but not used)
+            pos = t + stride < num_tiles ? advance_tile(p, pos, t + stride) : locate_tile(p, 0u);
             const uint64_t i_next = first_elem(pos);
             const uint32_t tag_next = p.view[pos.v].stream_tag;
             ok = mbar_wait(&acc_full[b], (it / kAccBufs) & 1, abort_flag);
             ok = __all_sync(0xffffffffu, ok);
             if (!ok) break;
             tc_fence_after_sync();
-            const uint32_t taddr = tmem_base + ((uint32_t)(q * 32) << 16) + b * kTile + half * 64;
-            uint32_t raw[32], n0[8], n1[8], packed[4], sb0 = 0, sb1 = 0;
-            float y[32];
-            // ---- first MX block
-            tmem_ld_32x32b_x32(taddr, raw);
-            tmem_ld_wait();
-            if (MODE == kModeSR) sr_draws32(p.keys, tag_next, i_next, n0);
+            const uint32_t taddr = tmem_base + ((uint32_t)(q * 32) << 16) + b * kTile;
+            uint32_t sb_all = 0;
 #pragma unroll
-            for (int i = 0; i < 32; ++i) y[i] = __uint_as_float(raw[i]) * cg;   // exact no-op unless g is 32 or 128
-            if (MODE == kModeDump) {
-                if (live) {
-                    float4* dst = reinterpret_cast<float4*>(y_dst);
-#pragma unroll
-                    for (int i = 0; i < 8; ++i) dst[i] = make_float4(y[4 * i], y[4 * i + 1], y[4 * i + 2], y[4 * i + 3]);
+            for (int j = 0; j < 4; ++j) {
+                uint32_t raw[32], nx[8], packed[4], sb = 0;
+                float y[32];
+                tmem_ld_32x32b_x32(taddr + 32 * j, raw);
+                tmem_ld_wait();
+                if (j == 3) {                                   // the accumulator is free once it has been read
+                    tc_fence_before_sync();
+                    __syncwarp();
+                    if (lane == 0) mbar_arrive(&acc_empty[b]);
                 }
-            } else {
-                quantize_block32_rw<MODE>(y, rw0, packed, sb0, p.pipe);
-                if (live) *reinterpret_cast<uint4*>(code_dst) = make_uint4(packed[0], packed[1], packed[2], packed[3]);
-            }
-            // ---- second MX block; the accumulator is free once it has been read
-            tmem_ld_32x32b_x32(taddr + 32, raw);
-            tmem_ld_wait();
-            tc_fence_before_sync();
-            __syncwarp();
-            if (lane == 0) mbar_arrive(&acc_empty[b]);
-            if (MODE == kModeSR) sr_draws32(p.keys, tag_next, i_next + 32, n1);
-#pragma unroll
-            for (int i = 0; i < 32; ++i) y[i] = __uint_as_float(raw[i]) * cg;
-            if (MODE == kModeDump) {
-                if (live) {
-                    float4* dst = reinterpret_cast<float4*>(y_dst + 32);
-#pragma unroll
-                    for (int i = 0; i < 8; ++i) dst[i] = make_float4(y[4 * i], y[4 * i + 1], y[4 * i + 2], y[4 * i + 3]);
+                if (MODE == kModeSR) {
+                    if (j < 3) sr_draws32(p.keys, tag_cur, i_cur + 32 * (j + 1), nx);
+                    else sr_draws32(p.keys, tag_next, i_next, nx);
                 }
-            } else {
-                quantize_block32_rw<MODE>(y, rw1, packed, sb1, p.pipe);
-                if (live) {
-                    *reinterpret_cast<uint4*>(code_dst + 16) = make_uint4(packed[0], packed[1], packed[2], packed[3]);
-                    *reinterpret_cast<uint16_t*>(scale_dst) = (uint16_t)(sb0 | (sb1 << 8));
+#pragma unroll
+                for (int i = 0; i < 32; ++i) y[i] = __uint_as_float(raw[i]) * cg;   // exact no-op unless g is 32 or 128
+                if (MODE == kModeDump) {
+                    if (live) {
+                        float4* dst = reinterpret_cast<float4*>(y_dst + 32 * j);
+#pragma unroll
+                        for (int i = 0; i < 8; ++i) dst[i] = make_float4(y[4 * i], y[4 * i + 1], y[4 * i + 2], y[4 * i + 3]);
+                    }
+                } else {
+                    quantize_block32_rw<MODE>(y, rw, packed, sb, p.pipe);
+                    if (live) *reinterpret_cast<uint4*>(code_dst + 16 * j) = make_uint4(packed[0], packed[1], packed[2], packed[3]);
+                    sb_all |= sb << (8 * j);
+                }
+                if (MODE == kModeSR) {
+#pragma unroll
+                    for (int i = 0; i < 8; ++i) rw[i] = nx[i];
                 }
             }
-            if (MODE == kModeSR) {
-#pragma unroll
-                for (int i = 0; i < 8; ++i) { rw0[i] = n0[i]; rw1[i] = n1[i]; }
-            }
+            if (MODE != kModeDump && live)
+                *reinterpret_cast<uint32_t*>(scale_dst) = sb_all;       // four consecutive bytes in either scale layout
         }
         if (!ok && lane == 0) *abort_flag = 1;
     }
@@ -340,7 +345,8 @@ cudaError_t launch_quantize_tc_group(const QuantArgs* a, int n, bool dump_y, cud
         w.r_tiles = (uint32_t)((w.R + kTile - 1) / kTile);
         w.k_tiles = (uint32_t)(w.K / kTile);
         w.tile_begin = tiles;
-        tiles += w.r_tiles * w.k_tiles;
+        w.n_tiles = w.r_tiles * w.k_tiles;
+        tiles += w.n_tiles;
         w.reduce_dim = a[v].reduce_dim;
         w.stream_tag = a[v].stream_tag;
         w.codes = a[v].codes; w.scales = a[v].scales; w.y_out = a[v].y_out;
@@ -364,6 +370,12 @@ cudaError_t launch_quantize_tc_group(const QuantArgs* a, int n, bool dump_y, cud
     e = cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
     if (e != cudaSuccess) return e;
     const unsigned grid = tiles < (uint32_t)sms ? tiles : (unsigned)sms;
+    for (int v = 0; v < kQuantMaxViews; ++v) {              // the two epilogue groups step through the list by 2 * grid
+        QView& w = p.view[v];
+        w.minor_count = w.reduce_dim == 1 ? w.k_tiles : w.r_tiles;
+        w.d_major = (uint32_t)kEpiGroups * grid / w.minor_count;
+        w.d_minor = (uint32_t)kEpiGroups * grid % w.minor_count;
+    }
     if (dump_y)
         quantize_tc_kernel<kModeDump><<<grid, kThreadsQ, kSmemQ, stream>>>(maps, p);
     else if (a[0].rounding == 0)
