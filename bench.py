@@ -295,6 +295,18 @@ def run_gpu(args):
                            "frac_of_nominal_9pf": gemm_tflops / NOMINAL_FP4_TFLOPS}
         calls_ms = sum(v[0] for v in agg.values()) / k_roof * 1e3
 
+        # On-box ceiling of the FP4 tensor pipe (resident operands, no loads, no epilogue): ~25 ms burst, ~0.3 s sustained.
+        def ceiling(mma_per_pair):
+            a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            a.record(stream); fl = mx.mxfp4_fp4_ceiling(mma_per_pair); b.record(stream)
+            torch.cuda.synchronize()
+            return fl / (a.elapsed_time(b) * 1e-3) / 1e12
+        ceiling(32000)
+        ceil_burst, ceil_sust = ceiling(320000), ceiling(3200000)
+        kernels["fp4_ceiling"] = {"burst_TFLOP/s": ceil_burst, "sustained_TFLOP/s": ceil_sust,
+                                  "gemm_frac_of_burst": gemm_tflops / ceil_burst, "gemm_frac_of_sustained": gemm_tflops / ceil_sust,
+                                  "what": "back-to-back 256x256x64 pair MMAs on shared-memory-resident operands"}
+
     clocks = sampler.stop()
     ms_e2e, h2d, d2h = None, 0, 0
     if "e2e" in legs:

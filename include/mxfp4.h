@@ -152,6 +152,15 @@ MXFP4_API mxfp4_status mxfp4_linear_backward_static(const void* dY, const void* 
                                                     int64_t b, int64_t m, int64_t n, int g, int rounding, uint64_t seed,
                                                     void* dX, void* dW, int out_dtype, void* cuda_stream);
 
+/*
+ * Measurement aid, not part of the method (the paper has no counterpart): launches a kernel in which every CTA pair
+ * issues `mma_per_pair` (rounded up to a multiple of 32) back-to-back 256 x 256 x 64 block-scaled FP4 tensor-core
+ * instructions on operands resident in shared memory: no loads, no output.  *flop_out (HOST pointer) receives the
+ * floating-point operations the launch performs; time the launch with CUDA events on `cuda_stream` to obtain the
+ * on-box ceiling of the FP4 tensor pipe.  Errors: MXFP4_ERR_SHAPE, MXFP4_ERR_DEVICE, MXFP4_ERR_CUDA.
+ */
+MXFP4_API mxfp4_status mxfp4_fp4_ceiling(int64_t mma_per_pair, int64_t* flop_out, void* cuda_stream);
+
 /* Size in bytes of a scale tensor for an operand [rows, K] in the given layout (NATIVE is padded). */
 MXFP4_API size_t mxfp4_scale_bytes(int64_t rows, int64_t K, int sf_layout);
 

@@ -33,6 +33,8 @@ _lib.mxfp4_linear_backward.argtypes = [_vp, _vp, _vp, _i64, _i64, _i64, _int, _i
 _lib.mxfp4_linear_backward.restype = _int
 _lib.mxfp4_linear_backward_static.argtypes = [_vp, _vp, _vp, _i64, _i64, _i64, _int, _int, _u64, _vp, _vp, _int, _vp]
 _lib.mxfp4_linear_backward_static.restype = _int
+_lib.mxfp4_fp4_ceiling.argtypes = [_i64, C.POINTER(C.c_int64), _vp]
+_lib.mxfp4_fp4_ceiling.restype = _int
 _lib.mxfp4_scale_bytes.argtypes = [_i64, _i64, _int]
 _lib.mxfp4_scale_bytes.restype = _sz
 _lib.mxfp4_device_status.argtypes = [_vp]
@@ -41,7 +43,8 @@ _lib.mxfp4_status_string.argtypes = [_int]
 _lib.mxfp4_status_string.restype = C.c_char_p
 
 EXPORTS = ["mxfp4_rht_sr_quantize", "mxfp4_rht", "mxfp4_gemm", "mxfp4_linear_backward_workspace",
-           "mxfp4_linear_backward", "mxfp4_linear_backward_static", "mxfp4_scale_bytes", "mxfp4_device_status", "mxfp4_status_string"]
+           "mxfp4_linear_backward", "mxfp4_linear_backward_static", "mxfp4_scale_bytes", "mxfp4_device_status", "mxfp4_status_string",
+           "mxfp4_fp4_ceiling"]
 
 
 class MxFp4Error(RuntimeError):
@@ -154,6 +157,13 @@ def mxfp4_linear_backward_static(dY, X, W, g: int, seed: int, rounding: int = RO
     _check(_lib.mxfp4_linear_backward_static(_ptr(dY), _ptr(X), _ptr(W), b, m, n, g, rounding, seed, _ptr(dX), _ptr(dW),
                                              out_dtype, _stream()))
     return dX, dW
+
+
+def mxfp4_fp4_ceiling(mma_per_pair: int) -> int:
+    """Launches the tensor-pipe ceiling kernel on the current stream and returns the flop it performs (time it with events)."""
+    flop = C.c_int64(0)
+    _check(_lib.mxfp4_fp4_ceiling(mma_per_pair, C.byref(flop), _stream()))
+    return int(flop.value)
 
 
 def mxfp4_device_status() -> int:

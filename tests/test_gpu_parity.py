@@ -235,3 +235,16 @@ def test_linear_backward_single_layer(gpu, ref, rounding):
     dXb, dWb = gpu.mxfp4_linear_backward(_dev(dY), _dev(X), _dev(W), 64, 0, rounding, gpu.OUT_BF16)
     assert np.linalg.norm(dXb.float().cpu().numpy() - dX) / np.linalg.norm(dX) <= 2.0 ** -8
     assert np.linalg.norm(dWb.float().cpu().numpy() - dW) / np.linalg.norm(dW) <= 2.0 ** -8
+
+
+# ------------------------------------------------------------------------------------- measurement aid
+
+def test_fp4_ceiling_kernel_runs_and_reports_its_work(gpu):
+    """The tensor-pipe ceiling kernel: flop count = pairs x MMAs (rounded up to 32) x 2*256*256*64, no timeout."""
+    import torch
+    pairs = torch.cuda.get_device_properties(0).multi_processor_count // 2
+    assert gpu.mxfp4_fp4_ceiling(40) == pairs * 64 * 2 * 256 * 256 * 64
+    assert gpu.mxfp4_fp4_ceiling(1) == pairs * 32 * 2 * 256 * 256 * 64
+    assert gpu.mxfp4_device_status() == 0
+    with pytest.raises(gpu.MxFp4Error):
+        gpu.mxfp4_fp4_ceiling(0)
