@@ -1,0 +1,59 @@
+"""The autograd wrapper: its gradients are the library's Algorithm-3 outputs, and they estimate the true gradients."""
+import numpy as np
+import pytest
+
+pytestmark = pytest.mark.gpu
+
+
+@pytest.fixture(scope="module")
+def torch_gpu():
+    import torch
+    if not torch.cuda.is_available():
+        pytest.skip("no GPU")
+    return torch
+
+
+def test_backward_is_the_library_call_and_estimates_the_gradient(torch_gpu):
+    torch = torch_gpu
+    from paper_2502_20586_b200 import binding as mx
+    from paper_2502_20586_b200.autograd import MxFp4Linear
+    gen = torch.Generator(device="cuda").manual_seed(3)
+    layer = MxFp4Linear(256, 384, g=64, seed=11)
+    x = torch.randn(4, 128, 256, device="cuda", generator=gen).to(torch.bfloat16).requires_grad_(True)
+    dy = (torch.randn(4, 128, 384, device="cuda", generator=gen) * 1e-3).to(torch.bfloat16)
+    y = layer(x)
+    assert y.shape == (4, 128, 384) and y.dtype == torch.bfloat16
+    y.backward(dy)
+    # identical to calling the library directly with the same seed
+    dx_lib, dw_lib = mx.mxfp4_linear_backward(dy.reshape(-1, 384), x.detach().reshape(-1, 256), layer.weight.detach(), 64, 11)
+    assert torch.equal(x.grad.reshape(-1, 256), dx_lib) and torch.equal(layer.weight.grad, dw_lib)
+    # and a reasonable one-sample estimate of the exact gradients
+    dx_ref = dy.double().reshape(-1, 384) @ layer.weight.detach().double()
+    dw_ref = dy.double().reshape(-1, 384).t() @ x.detach().double().reshape(-1, 256)
+    ex = float((x.grad.double().reshape(-1, 256) - dx_ref).norm() / dx_ref.norm())
+    ew = float((layer.weight.grad.double() - dw_ref).norm() / dw_ref.norm())
+    assert ex < 0.5 and ew < 0.5
+    assert mx.mxfp4_device_status() == 0
+
+
+def test_seeds_advance_and_the_mean_gradient_converges(torch_gpu):
+    """SR makes the backward unbiased (Lemma 3.1): the mean over T calls approaches the exact gradient like T^-1/2."""
+    torch = torch_gpu
+    from paper_2502_20586_b200.autograd import MxFp4Linear
+    gen = torch.Generator(device="cuda").manual_seed(5)
+    layer = MxFp4Linear(128, 128, g=32, seed=100)
+    x = torch.randn(256, 128, device="cuda", generator=gen).to(torch.bfloat16)
+    dy = (torch.randn(256, 128, device="cuda", generator=gen) * 1e-2).to(torch.bfloat16)
+    dw_ref = dy.double().t() @ x.double()
+    T = 64
+    acc = torch.zeros_like(dw_ref)
+    first = None
+    for _ in range(T):
+        layer.weight.grad = None
+        layer(x).backward(dy)
+        acc += layer.weight.grad.double()
+        if first is None:
+            first = float((layer.weight.grad.double() - dw_ref).norm() / dw_ref.norm())
+    mean_err = float((acc / T - dw_ref).norm() / dw_ref.norm())
+    assert layer.calls == T
+    assert mean_err < first / 4          # ideal: first / 8
