@@ -425,6 +425,18 @@ ORC_API int orc_linear_backward(const uint16_t *dY, const uint16_t *X, const uin
     return rc;
 }
 
+/* Bias gradient of the linear layer y = x W^T + b (problem statement, Section 2: dL/db = 1 dL/dy): the column sums
+ * of dY [b, m], computed exactly as a plain loop in fp64 (bf16 inputs are exact in fp64; 2^14 terms lose nothing
+ * that matters).  Not quantised: the paper's recipe touches only the two matrix products. */
+ORC_API void orc_bias_grad(const uint16_t *dY, int64_t b, int64_t m, double *db)
+{
+    for (int64_t j = 0; j < m; ++j) {
+        double s = 0.0;
+        for (int64_t i = 0; i < b; ++i) s += bf16_to_double(dY[i * m + j]);
+        db[j] = s;
+    }
+}
+
 ORC_API int orc_num_threads(void)
 {
 #ifdef _OPENMP

@@ -56,6 +56,8 @@ _lib.orc_linear_backward.argtypes = [_u16p, _u16p, _u16p, _i64, _i64, _i64, C.c_
                                      C.c_void_p, _i64, C.c_void_p, _i64,
                                      C.c_void_p, _i64, C.c_void_p, _i64, _f64p, _f64p]
 _lib.orc_linear_backward.restype = C.c_int
+_lib.orc_bias_grad.argtypes = [_u16p, _i64, _i64, _f64p]
+_lib.orc_bias_grad.restype = None
 _lib.orc_num_threads.argtypes = []
 _lib.orc_num_threads.restype = C.c_int
 
@@ -191,6 +193,14 @@ def gemm_bf16(A, B, rows=None, cols=None, a_transpose=False, b_transpose=False) 
     out = np.empty((nr, nc), np.float64)
     _lib.orc_gemm_bf16(ap, asr, ask, bp, bsr, bsk, K, rp, nr, cp, nc, out)
     return out
+
+
+def bias_grad(dY):
+    """dL/db = column sums of bf16 dY [b, m], fp64 (problem statement, Section 2)."""
+    b, m = dY.shape
+    db = np.empty(m, np.float64)
+    _lib.orc_bias_grad(dY, b, m, db)
+    return db
 
 
 def linear_backward(dY, X, W, g, rounding, seed, dx_rows=None, dx_cols=None, dw_rows=None, dw_cols=None):

@@ -421,3 +421,22 @@ def test_sr_gemm_variance_formula_and_rht_trend(ref):
         return tot / trials
     assert mean_var(0.1, True) < mean_var(0.1, False)
     assert abs(mean_var(0.0, True) / mean_var(0.0, False) - 1.0) < 0.25
+
+
+def test_bias_grad_closed_forms(ref):
+    """dL/db = 1 dL/dy (problem statement): closed forms a transposed index, a dropped row or a wrong stride would break."""
+    b, m = 96, 40
+    # dY[i, j] = j + 1: every column sums to b (j + 1)
+    dY = np.tile(np.arange(1, m + 1, dtype=np.float64), (b, 1))
+    assert np.array_equal(ref.bias_grad(wl.to_bf16_bits(dY)), b * np.arange(1, m + 1, dtype=np.float64))
+    # dY[i, j] = i for j == 3 only: Gauss sum in one column, zeros elsewhere
+    dY = np.zeros((b, m)); dY[:, 3] = np.arange(b)
+    want = np.zeros(m); want[3] = b * (b - 1) / 2
+    assert np.array_equal(ref.bias_grad(wl.to_bf16_bits(dY)), want)
+    # alternating signs cancel exactly; a lone last row survives
+    dY = np.ones((b + 1, m)); dY[1::2] = -1.0; dY[-1] = 0.25
+    assert np.array_equal(ref.bias_grad(wl.to_bf16_bits(dY)), np.full(m, 0.25))
+    # random bf16 data against numpy's own sum of the exactly converted values
+    rng = np.random.default_rng(7)
+    bits = wl.to_bf16_bits(rng.standard_normal((300, 24)) * 1e-3)
+    np.testing.assert_allclose(ref.bias_grad(bits), wl.bf16_bits_to_f64(bits).sum(axis=0), rtol=1e-13, atol=0)
