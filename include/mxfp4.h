@@ -128,6 +128,21 @@ MXFP4_API mxfp4_status mxfp4_linear_backward(const void* dY, const void* X, cons
                                    void* workspace, size_t workspace_bytes, void* cuda_stream);
 
 /*
+ * Algorithm 3 with the two remaining pieces of a linear layer's backward (problem statement, Section 2:
+ * dL/db = 1 dL/dy; micro-batch gradient accumulation):
+ *   db:         NULL, or fp32 [m] (16-byte aligned): the bias gradient, column sums of dY in fp32 (not quantised).
+ *   accumulate: 0: dW = ..., db = ...;  1: dW += ..., db += ... (out_dtype must be MXFP4_OUT_FP32, else
+ *               MXFP4_ERR_MODE).  dX is overwritten in both cases.
+ *   workspace:  at least mxfp4_linear_backward_ex_workspace(b, m, n, db != NULL) bytes, 256-byte aligned.
+ * Everything else as mxfp4_linear_backward.
+ */
+MXFP4_API size_t mxfp4_linear_backward_ex_workspace(int64_t b, int64_t m, int64_t n, int with_bias);
+MXFP4_API mxfp4_status mxfp4_linear_backward_ex(const void* dY, const void* X, const void* W,
+                                      int64_t b, int64_t m, int64_t n, int g, int rounding, uint64_t seed,
+                                      void* dX, void* dW, float* db, int out_dtype, int accumulate,
+                                      void* workspace, size_t workspace_bytes, void* cuda_stream);
+
+/*
  * The same backward pass for callers that cannot supply a workspace.  (The paper has no counterpart: this is a
  * property of the library, not of the method.)
  *

@@ -33,6 +33,10 @@ _lib.mxfp4_linear_backward.argtypes = [_vp, _vp, _vp, _i64, _i64, _i64, _int, _i
 _lib.mxfp4_linear_backward.restype = _int
 _lib.mxfp4_linear_backward_static.argtypes = [_vp, _vp, _vp, _i64, _i64, _i64, _int, _int, _u64, _vp, _vp, _int, _vp]
 _lib.mxfp4_linear_backward_static.restype = _int
+_lib.mxfp4_linear_backward_ex_workspace.argtypes = [_i64, _i64, _i64, _int]
+_lib.mxfp4_linear_backward_ex_workspace.restype = _sz
+_lib.mxfp4_linear_backward_ex.argtypes = [_vp, _vp, _vp, _i64, _i64, _i64, _int, _int, _u64, _vp, _vp, _vp, _int, _int, _vp, _sz, _vp]
+_lib.mxfp4_linear_backward_ex.restype = _int
 _lib.mxfp4_fp4_ceiling.argtypes = [_i64, C.POINTER(C.c_int64), _vp]
 _lib.mxfp4_fp4_ceiling.restype = _int
 _lib.mxfp4_scale_bytes.argtypes = [_i64, _i64, _int]
@@ -44,7 +48,7 @@ _lib.mxfp4_status_string.restype = C.c_char_p
 
 EXPORTS = ["mxfp4_rht_sr_quantize", "mxfp4_rht", "mxfp4_gemm", "mxfp4_linear_backward_workspace",
            "mxfp4_linear_backward", "mxfp4_linear_backward_static", "mxfp4_scale_bytes", "mxfp4_device_status", "mxfp4_status_string",
-           "mxfp4_fp4_ceiling"]
+           "mxfp4_fp4_ceiling", "mxfp4_linear_backward_ex_workspace", "mxfp4_linear_backward_ex"]
 
 
 class MxFp4Error(RuntimeError):
@@ -135,6 +139,32 @@ def mxfp4_linear_backward(dY, X, W, g: int, seed: int, rounding: int = ROUND_SR,
     _check(_lib.mxfp4_linear_backward(_ptr(dY), _ptr(X), _ptr(W), b, m, n, g, rounding, seed, _ptr(dX), _ptr(dW),
                                       out_dtype, _ptr(workspace), workspace.numel(), _stream()))
     return dX, dW
+
+
+def mxfp4_linear_backward_ex(dY, X, W, g: int, seed: int, rounding: int = ROUND_SR, out_dtype: int = OUT_BF16,
+                             dX=None, dW=None, db=None, with_bias: bool = False, accumulate: bool = False, workspace=None):
+    """Algorithm 3 plus the bias gradient (fp32 [m], column sums of dY) and accumulation into fp32 dW / db.
+    Returns (dX, dW, db) with db None unless with_bias or db is given."""
+    b, m = dY.shape
+    _, n = X.shape
+    for t in (dY, X, W):
+        assert t.is_cuda and t.dtype == torch.bfloat16 and t.is_contiguous()
+    dt = torch.float32 if out_dtype == OUT_FP32 else torch.bfloat16
+    if dX is None:
+        dX = torch.empty((b, n), dtype=dt, device=dY.device)
+    if dW is None:
+        assert not accumulate, "accumulation needs an existing dW"
+        dW = torch.empty((m, n), dtype=dt, device=dY.device)
+    if db is None and with_bias:
+        assert not accumulate, "accumulation needs an existing db"
+        db = torch.empty((m,), dtype=torch.float32, device=dY.device)
+    need = int(_lib.mxfp4_linear_backward_ex_workspace(b, m, n, 1 if db is not None else 0))
+    if workspace is None:
+        workspace = torch.empty(need, dtype=torch.uint8, device=dY.device)
+    _check(_lib.mxfp4_linear_backward_ex(_ptr(dY), _ptr(X), _ptr(W), b, m, n, g, rounding, seed, _ptr(dX), _ptr(dW),
+                                         _ptr(db) if db is not None else None, out_dtype, 1 if accumulate else 0,
+                                         _ptr(workspace), workspace.numel(), _stream()))
+    return dX, dW, db
 
 
 STATIC_WORKSPACE_BYTES = 8 << 20

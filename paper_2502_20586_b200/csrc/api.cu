@@ -148,7 +148,8 @@ bool make_output_map(CUtensorMap* map, void* C, int64_t M, int64_t N, int64_t ld
 }
 
 mxfp4_status gemm_impl(const uint8_t* A_codes, const uint8_t* A_scales, const uint8_t* B_codes, const uint8_t* B_scales, int64_t M,
-                       int64_t N, int64_t K, float alpha, void* C, int64_t ldc, int out_dtype, cudaStream_t stream) {
+                       int64_t N, int64_t K, float alpha, void* C, int64_t ldc, int out_dtype, cudaStream_t stream,
+                       int accumulate = 0) {
     GemmArgs a;
     mxfp4_status st = make_codes_map(&a.tmap_a, A_codes, M, K, mx::kGemmBM);
     if (st != MXFP4_OK) return st;
@@ -157,6 +158,7 @@ mxfp4_status gemm_impl(const uint8_t* A_codes, const uint8_t* A_scales, const ui
     a.sfa = A_scales; a.sfb = B_scales;
     a.M = M; a.N = N; a.K = K;
     a.alpha = alpha; a.C = C; a.ldc = ldc; a.out_fp32 = out_dtype == MXFP4_OUT_FP32;
+    a.accumulate = accumulate;
     a.use_pair = g_rt.gemm_pair && M > 128;                   // one 128-row tile gives a pair nothing to share
     if (a.use_pair) {
         st = make_codes_map(&a.tmap_b_half, B_codes, N, K, 128);
@@ -253,9 +255,13 @@ size_t mxfp4_linear_backward_workspace(int64_t b, int64_t m, int64_t n) {
     return plan_workspace(b, m, n).total;
 }
 
-mxfp4_status mxfp4_linear_backward(const void* dY, const void* X, const void* W, int64_t b, int64_t m, int64_t n, int g, int rounding,
-                                   uint64_t seed, void* dX, void* dW, int out_dtype, void* workspace, size_t workspace_bytes,
-                                   void* cuda_stream) {
+}  // extern "C"
+
+namespace {
+// Algorithm 3, optionally with the bias gradient (db != NULL) and accumulation into dW and db.
+mxfp4_status linear_backward_impl(const void* dY, const void* X, const void* W, int64_t b, int64_t m, int64_t n, int g, int rounding,
+                                  uint64_t seed, void* dX, void* dW, float* db, int out_dtype, int accumulate, void* workspace,
+                                  size_t workspace_bytes, void* cuda_stream) {
     if (!dY || !X || !W || !dX || !dW) return MXFP4_ERR_NULL;
     if (b <= 0 || m <= 0 || n <= 0) return MXFP4_ERR_SHAPE;
     if (!valid_g(g)) return MXFP4_ERR_BAD_G;
@@ -263,8 +269,12 @@ mxfp4_status mxfp4_linear_backward(const void* dY, const void* X, const void* W,
     if (g != 0 && (m % g != 0 || b % g != 0)) return MXFP4_ERR_BAD_G;
     if (rounding != MXFP4_ROUND_SR && rounding != MXFP4_ROUND_RN) return MXFP4_ERR_MODE;
     if (out_dtype != MXFP4_OUT_BF16 && out_dtype != MXFP4_OUT_FP32) return MXFP4_ERR_MODE;
-    if (!aligned16(dY) || !aligned16(X) || !aligned16(W) || !aligned16(dX) || !aligned16(dW)) return MXFP4_ERR_ALIGN;
-    const Workspace ws = plan_workspace(b, m, n);
+    if (accumulate != 0 && accumulate != 1) return MXFP4_ERR_MODE;
+    if (accumulate == 1 && out_dtype != MXFP4_OUT_FP32) return MXFP4_ERR_MODE;      // accumulation is defined on fp32 gradients
+    if (!aligned16(dY) || !aligned16(X) || !aligned16(W) || !aligned16(dX) || !aligned16(dW) || (db && !aligned16(db))) return MXFP4_ERR_ALIGN;
+    Workspace ws = plan_workspace(b, m, n);
+    const size_t bias_off = ws.total;
+    if (db != nullptr) ws.total += (size_t)round_up((int64_t)mx::bias_grad_workspace(b, m), 1024);
     if (workspace == nullptr || workspace_bytes < ws.total || (reinterpret_cast<uintptr_t>(workspace) & 255u) != 0) return MXFP4_ERR_WORKSPACE;
     mxfp4_status st = runtime_init();
     if (st != MXFP4_OK) return st;
@@ -297,13 +307,36 @@ mxfp4_status mxfp4_linear_backward(const void* dY, const void* X, const void* W,
     ForkJoin* fj = ws.total > (size_t)MXFP4_STATIC_WORKSPACE_BYTES && waves_dx >= 74 && waves_dw >= 74 ? fork_join() : nullptr;
     if (fj != nullptr && (cudaEventRecord(fj->fork, stream) != cudaSuccess || cudaStreamWaitEvent(fj->side, fj->fork, 0) != cudaSuccess))
         return MXFP4_ERR_CUDA;
-    st = gemm_impl(c[0], s[0], c[1], s[1], b, n, m, alpha, dX, n, out_dtype, stream);
+    st = gemm_impl(c[0], s[0], c[1], s[1], b, n, m, alpha, dX, n, out_dtype, stream);      // dX is never accumulated
     if (st != MXFP4_OK) return st;
-    st = gemm_impl(c[2], s[2], c[3], s[3], m, n, b, alpha, dW, n, out_dtype, fj != nullptr ? fj->side : stream);
+    st = gemm_impl(c[2], s[2], c[3], s[3], m, n, b, alpha, dW, n, out_dtype, fj != nullptr ? fj->side : stream, accumulate);
     if (st != MXFP4_OK) return st;
+    // dL/db = 1 dL/dy (problem statement): column sums of dY, after the GEMMs on the caller's stream
+    if (db != nullptr && mx::launch_bias_grad(dY, b, m, m, accumulate, db, reinterpret_cast<float*>(base + bias_off), stream) != cudaSuccess)
+        return MXFP4_ERR_CUDA;
     if (fj != nullptr && (cudaEventRecord(fj->join, fj->side) != cudaSuccess || cudaStreamWaitEvent(stream, fj->join, 0) != cudaSuccess))
         return MXFP4_ERR_CUDA;
     return MXFP4_OK;
+}
+}  // namespace
+
+extern "C" {
+
+mxfp4_status mxfp4_linear_backward(const void* dY, const void* X, const void* W, int64_t b, int64_t m, int64_t n, int g, int rounding,
+                                   uint64_t seed, void* dX, void* dW, int out_dtype, void* workspace, size_t workspace_bytes,
+                                   void* cuda_stream) {
+    return linear_backward_impl(dY, X, W, b, m, n, g, rounding, seed, dX, dW, nullptr, out_dtype, 0, workspace, workspace_bytes, cuda_stream);
+}
+
+size_t mxfp4_linear_backward_ex_workspace(int64_t b, int64_t m, int64_t n, int with_bias) {
+    if (b <= 0 || m <= 0 || n <= 0) return 0;
+    return plan_workspace(b, m, n).total + (with_bias ? (size_t)round_up((int64_t)mx::bias_grad_workspace(b, m), 1024) : 0);
+}
+
+mxfp4_status mxfp4_linear_backward_ex(const void* dY, const void* X, const void* W, int64_t b, int64_t m, int64_t n, int g, int rounding,
+                                      uint64_t seed, void* dX, void* dW, float* db, int out_dtype, int accumulate, void* workspace,
+                                      size_t workspace_bytes, void* cuda_stream) {
+    return linear_backward_impl(dY, X, W, b, m, n, g, rounding, seed, dX, dW, db, out_dtype, accumulate, workspace, workspace_bytes, cuda_stream);
 }
 
 mxfp4_status mxfp4_device_status(void* cuda_stream) {

@@ -48,6 +48,7 @@ struct Params {
     int64_t M, N, K, ldc;
     float alpha;
     int out_fp32;
+    int accumulate;                                         // fp32 output only: C += instead of C =
     int m_tiles, n_tiles;
 };
 
@@ -211,10 +212,15 @@ gemm_mxf4_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_consta
                         float* dst = static_cast<float*>(p.C) + row * p.ldc + col;
 #pragma unroll
                         for (int v = 0; v < 8; ++v)
-                            if (4 * v < nvalid)
-                                reinterpret_cast<float4*>(dst)[v] =
-                                    make_float4(__uint_as_float(r[4 * v]) * p.alpha, __uint_as_float(r[4 * v + 1]) * p.alpha,
-                                                __uint_as_float(r[4 * v + 2]) * p.alpha, __uint_as_float(r[4 * v + 3]) * p.alpha);
+                            if (4 * v < nvalid) {
+                                float4 o = p.accumulate ? reinterpret_cast<const float4*>(dst)[v] : make_float4(0.f, 0.f, 0.f, 0.f);
+                                // product rounded first, then one add: the same two roundings as the TMA-reduce path (no fused multiply-add)
+                                o.x = __fadd_rn(o.x, __fmul_rn(__uint_as_float(r[4 * v]), p.alpha));
+                                o.y = __fadd_rn(o.y, __fmul_rn(__uint_as_float(r[4 * v + 1]), p.alpha));
+                                o.z = __fadd_rn(o.z, __fmul_rn(__uint_as_float(r[4 * v + 2]), p.alpha));
+                                o.w = __fadd_rn(o.w, __fmul_rn(__uint_as_float(r[4 * v + 3]), p.alpha));
+                                reinterpret_cast<float4*>(dst)[v] = o;
+                            }
                     } else {
                         __nv_bfloat16* dst = static_cast<__nv_bfloat16*>(p.C) + row * p.ldc + col;
 #pragma unroll
@@ -262,7 +268,7 @@ cudaError_t launch_gemm(const GemmArgs& a, cudaStream_t stream) {
     Params p;
     p.sfa = a.sfa; p.sfb = a.sfb; p.C = a.C;
     p.M = a.M; p.N = a.N; p.K = a.K; p.ldc = a.ldc;
-    p.alpha = a.alpha; p.out_fp32 = a.out_fp32;
+    p.alpha = a.alpha; p.out_fp32 = a.out_fp32; p.accumulate = a.accumulate;
     p.m_tiles = (int)((a.M + BM - 1) / BM);
     p.n_tiles = (int)((a.N + BN - 1) / BN);
     int dev = 0, sms = 0;

@@ -52,6 +52,7 @@ struct ParamsP {
     int out_fp32;
     int m_tiles, n_tiles;                                   // in pair tiles
     int c_tma;                                              // C goes out through tmap_c (else plain stores)
+    int accumulate;                                         // fp32 output only: C += instead of C =
 };
 
 __device__ __forceinline__ void tile_coords_p(int t, int m_tiles, int n_tiles, int& mt, int& nt) {
@@ -257,7 +258,10 @@ gemm_mxf4_pair_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_c
             fence_proxy_async_smem();
             __syncwarp();
             if (lane == 0) {
-                if (in_range) tma_store_2d(&tmap_c, buf, col, row0);
+                if (in_range) {
+                    if (p.accumulate) tma_reduce_add_2d(&tmap_c, buf, col, row0);
+                    else tma_store_2d(&tmap_c, buf, col, row0);
+                }
                 bulk_commit_group();
             }
             ++n_stores;
@@ -338,10 +342,15 @@ gemm_mxf4_pair_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_c
                         float* dst = static_cast<float*>(p.C) + row * p.ldc + col;
 #pragma unroll
                         for (int v = 0; v < 8; ++v)
-                            if (4 * v < nvalid)
-                                reinterpret_cast<float4*>(dst)[v] =
-                                    make_float4(__uint_as_float(r[4 * v]) * p.alpha, __uint_as_float(r[4 * v + 1]) * p.alpha,
-                                                __uint_as_float(r[4 * v + 2]) * p.alpha, __uint_as_float(r[4 * v + 3]) * p.alpha);
+                            if (4 * v < nvalid) {
+                                float4 o = p.accumulate ? reinterpret_cast<const float4*>(dst)[v] : make_float4(0.f, 0.f, 0.f, 0.f);
+                                // product rounded first, then one add: the same two roundings as the TMA-reduce path (no fused multiply-add)
+                                o.x = __fadd_rn(o.x, __fmul_rn(__uint_as_float(r[4 * v]), p.alpha));
+                                o.y = __fadd_rn(o.y, __fmul_rn(__uint_as_float(r[4 * v + 1]), p.alpha));
+                                o.z = __fadd_rn(o.z, __fmul_rn(__uint_as_float(r[4 * v + 2]), p.alpha));
+                                o.w = __fadd_rn(o.w, __fmul_rn(__uint_as_float(r[4 * v + 3]), p.alpha));
+                                reinterpret_cast<float4*>(dst)[v] = o;
+                            }
                     } else {
                         __nv_bfloat16* dst = static_cast<__nv_bfloat16*>(p.C) + row * p.ldc + col;
 #pragma unroll
@@ -398,6 +407,7 @@ cudaError_t launch_gemm_pair(const GemmArgs& a, cudaStream_t stream) {
     const int tiles = p.m_tiles * p.n_tiles;
     const int pairs = tiles < sms / 2 ? tiles : sms / 2;
     p.c_tma = a.has_tmap_c ? 1 : 0;
+    p.accumulate = a.accumulate;
     gemm_mxf4_pair_kernel<<<2 * pairs, kThreadsP, kSmemP, stream>>>(a.tmap_a, a.tmap_b_half, a.tmap_c, p);
     return cudaGetLastError();
 }

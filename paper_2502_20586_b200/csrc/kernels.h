@@ -47,11 +47,17 @@ struct GemmArgs {
     void* C;
     int64_t ldc;
     int out_fp32;
+    int accumulate;       // C += alpha A B^T instead of C = (fp32 output only)
 };
 
 constexpr int kGemmBM = 128;
 constexpr int kGemmBN = 256;
 constexpr int kGemmBKBytes = 128;   // 256 E2M1 elements per pipeline stage
+
+// Bias gradient: db [m] (fp32) = (accumulate ? db : 0) + column sums of bf16 dY [b, m]; `partial` is scratch of
+// bias_grad_workspace(b, m) bytes.
+size_t bias_grad_workspace(int64_t b, int64_t m);
+cudaError_t launch_bias_grad(const void* dY, int64_t b, int64_t m, int64_t ld, int accumulate, float* db, float* partial, cudaStream_t stream);
 
 cudaError_t launch_gemm(const GemmArgs& a, cudaStream_t stream);
 cudaError_t gemm_init();            // one-time: opt in to large dynamic shared memory

@@ -2,7 +2,7 @@
 
     python -m paper_2502_20586_b200.microbench gemm  M N K            [--iters 20] [--out fp32]
     python -m paper_2502_20586_b200.microbench quant ROWS COLS REDUCE_DIM G [--rounding 0] [--iters 20]
-    python -m paper_2502_20586_b200.microbench backward B N M G       [--iters 20]
+    python -m paper_2502_20586_b200.microbench backward B N M G       [--iters 20] [--bias] [--accumulate --out fp32]
 
 Operands are random codes/scales (gemm) or N(0,1) bf16 (quant, backward).  Between timed launches a buffer
 larger than L2 is rewritten so every launch starts with a cold L2.  Prints one JSON line.
@@ -45,6 +45,8 @@ def main(argv=None):
     ap.add_argument("--rounding", type=int, default=0)
     ap.add_argument("--out", default="bf16")
     ap.add_argument("--no-flush", action="store_true")
+    ap.add_argument("--bias", action="store_true", help="backward: also the bias gradient (extended entry point)")
+    ap.add_argument("--accumulate", action="store_true", help="backward: accumulate into fp32 dW / db")
     args = ap.parse_args(argv)
     dev = torch.device("cuda", 0)
     torch.cuda.set_device(dev)
@@ -77,11 +79,18 @@ def main(argv=None):
         dY = torch.randn((b, m), generator=gen, device=dev).to(torch.bfloat16)
         X = torch.randn((b, n), generator=gen, device=dev).to(torch.bfloat16)
         W = torch.randn((m, n), generator=gen, device=dev).to(torch.bfloat16)
-        dX = torch.empty((b, n), dtype=torch.bfloat16, device=dev)
-        dW = torch.empty((m, n), dtype=torch.bfloat16, device=dev)
-        ws = torch.empty(mx.mxfp4_linear_backward_workspace(b, m, n), dtype=torch.uint8, device=dev)
-        med, best = _time(lambda: mx.mxfp4_linear_backward(dY, X, W, g, 0, args.rounding, out_dtype, dX=dX, dW=dW, workspace=ws),
-                          args.iters, flush)
+        dt = torch.float32 if out_dtype == mx.OUT_FP32 else torch.bfloat16
+        dX = torch.empty((b, n), dtype=dt, device=dev)
+        dW = torch.zeros((m, n), dtype=dt, device=dev)
+        if args.bias or args.accumulate:
+            db = torch.zeros((m,), dtype=torch.float32, device=dev) if args.bias else None
+            ws = torch.empty(mx.mxfp4_linear_backward_workspace(b, m, n) + (64 * m * 4 + 1024), dtype=torch.uint8, device=dev)
+            fn = lambda: mx.mxfp4_linear_backward_ex(dY, X, W, g, 0, args.rounding, out_dtype, dX=dX, dW=dW, db=db,
+                                                     accumulate=args.accumulate, workspace=ws)
+        else:
+            ws = torch.empty(mx.mxfp4_linear_backward_workspace(b, m, n), dtype=torch.uint8, device=dev)
+            fn = lambda: mx.mxfp4_linear_backward(dY, X, W, g, 0, args.rounding, out_dtype, dX=dX, dW=dW, workspace=ws)
+        med, best = _time(fn, args.iters, flush)
         fl = 4.0 * b * m * n
         res.update(ms=med, ms_best=best, tflops=fl / med / 1e9, tflops_best=fl / best / 1e9)
     status = mx.mxfp4_device_status()

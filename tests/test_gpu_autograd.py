@@ -18,7 +18,7 @@ def test_backward_is_the_library_call_and_estimates_the_gradient(torch_gpu):
     from paper_2502_20586_b200 import binding as mx
     from paper_2502_20586_b200.autograd import MxFp4Linear
     gen = torch.Generator(device="cuda").manual_seed(3)
-    layer = MxFp4Linear(256, 384, g=64, seed=11)
+    layer = MxFp4Linear(256, 384, bias=True, g=64, seed=11)
     x = torch.randn(4, 128, 256, device="cuda", generator=gen).to(torch.bfloat16).requires_grad_(True)
     dy = (torch.randn(4, 128, 384, device="cuda", generator=gen) * 1e-3).to(torch.bfloat16)
     y = layer(x)
@@ -33,6 +33,9 @@ def test_backward_is_the_library_call_and_estimates_the_gradient(torch_gpu):
     ex = float((x.grad.double().reshape(-1, 256) - dx_ref).norm() / dx_ref.norm())
     ew = float((layer.weight.grad.double() - dw_ref).norm() / dw_ref.norm())
     assert ex < 0.5 and ew < 0.5
+    # the bias gradient is the plain column sum (bf16-rounded for the bf16 parameter)
+    db_ref = dy.double().reshape(-1, 384).sum(0)
+    assert float((layer.bias.grad.double() - db_ref).abs().max()) <= 2.0 ** -8 * float(db_ref.abs().max()) + 1e-12
     assert mx.mxfp4_device_status() == 0
 
 

@@ -248,3 +248,41 @@ def test_fp4_ceiling_kernel_runs_and_reports_its_work(gpu):
     assert gpu.mxfp4_device_status() == 0
     with pytest.raises(gpu.MxFp4Error):
         gpu.mxfp4_fp4_ceiling(0)
+
+
+# ------------------------------------------------------------------------------------- bias gradient, accumulation
+
+@pytest.mark.parametrize("b,m,n", [(256, 512, 512), (384, 640, 264), (2048, 1152, 128), (256, 128, 64)])
+def test_bias_grad_and_accumulation(gpu, ref, b, m, n):
+    """dL/db = 1 dL/dy in fp32 against the fp64 oracle; accumulate adds a second micro-batch into fp32 dW and db."""
+    import torch
+    rng = np.random.default_rng(b + m)
+    m = (m // 128) * 128
+    dY = wl.to_bf16_bits(rng.standard_t(3, (b, m)) * 1e-3)
+    X = wl.to_bf16_bits(rng.standard_normal((b, n)))
+    W = wl.to_bf16_bits(rng.standard_normal((m, n)) * 0.02)
+    dX, dW, db = gpu.mxfp4_linear_backward_ex(_dev(dY), _dev(X), _dev(W), 64, 5, gpu.ROUND_SR, gpu.OUT_FP32, with_bias=True)
+    assert gpu.mxfp4_device_status() == 0
+    # fp32 sums of b terms: error bounded by b 2^-24 sum|dY| per column; typical sqrt(b) 2^-24
+    want = ref.bias_grad(dY)
+    bound = 64 * np.sqrt(b) * 2.0 ** -24 * np.abs(wl.bf16_bits_to_f64(dY)).sum(axis=0) + 1e-30
+    assert np.all(np.abs(db.cpu().numpy().astype(np.float64) - want) <= bound)
+    # the other outputs equal the plain call's
+    dX0, dW0 = gpu.mxfp4_linear_backward(_dev(dY), _dev(X), _dev(W), 64, 5, gpu.ROUND_SR, gpu.OUT_FP32)
+    assert torch.equal(dX, dX0) and torch.equal(dW, dW0)
+    # second micro-batch with another seed, accumulated
+    dY2 = wl.to_bf16_bits(rng.standard_t(3, (b, m)) * 1e-3)
+    X2 = wl.to_bf16_bits(rng.standard_normal((b, n)))
+    _, dW1, _ = gpu.mxfp4_linear_backward_ex(_dev(dY2), _dev(X2), _dev(W), 64, 6, gpu.ROUND_SR, gpu.OUT_FP32)
+    dWa, dba = dW.clone(), db.clone()
+    dX2, dWa, dba = gpu.mxfp4_linear_backward_ex(_dev(dY2), _dev(X2), _dev(W), 64, 6, gpu.ROUND_SR, gpu.OUT_FP32,
+                                                  dW=dWa, db=dba, accumulate=True)
+    assert gpu.mxfp4_device_status() == 0
+    assert torch.equal(dWa, dW + dW1)                      # one fp32 add per element, same operands: exact
+    want2 = want + ref.bias_grad(dY2)
+    bound2 = bound + 64 * np.sqrt(b) * 2.0 ** -24 * np.abs(wl.bf16_bits_to_f64(dY2)).sum(axis=0)
+    assert np.all(np.abs(dba.cpu().numpy().astype(np.float64) - want2) <= bound2)
+    # bf16 output cannot accumulate
+    with pytest.raises(gpu.MxFp4Error):
+        gpu.mxfp4_linear_backward_ex(_dev(dY), _dev(X), _dev(W), 64, 5, gpu.ROUND_SR, gpu.OUT_BF16,
+                                     dW=torch.zeros((m, n), dtype=torch.bfloat16, device="cuda"), accumulate=True)
