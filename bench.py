@@ -295,6 +295,8 @@ def run_gpu(args):
                            "frac_of_nominal_9pf": gemm_tflops / NOMINAL_FP4_TFLOPS}
         calls_ms = sum(v[0] for v in agg.values()) / k_roof * 1e3
 
+    clocks = sampler.stop()
+    if gemm_tflops is not None:
         # On-box ceiling of the FP4 tensor pipe (resident operands, no loads, no epilogue): ~25 ms burst, ~0.3 s sustained.
         def ceiling(mma_per_pair):
             a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
@@ -306,8 +308,6 @@ def run_gpu(args):
         kernels["fp4_ceiling"] = {"burst_TFLOP/s": ceil_burst, "sustained_TFLOP/s": ceil_sust,
                                   "gemm_frac_of_burst": gemm_tflops / ceil_burst, "gemm_frac_of_sustained": gemm_tflops / ceil_sust,
                                   "what": "back-to-back 256x256x64 pair MMAs on shared-memory-resident operands"}
-
-    clocks = sampler.stop()
     ms_e2e, h2d, d2h = None, 0, 0
     if "e2e" in legs:
         # ---- e2e: host buffers, copies inside the timed region
