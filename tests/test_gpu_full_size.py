@@ -1,4 +1,4 @@
-"""Parity at the benchmark's full sizes (GPT 6.7B layer shapes, g = 128), in the launch configuration bench.py times.
+"""Parity at full sizes (GPT 345M / 1.3B / 6.7B layer shapes with their g), in the launch configuration bench.py times.
 
 The oracle cannot run whole 16384 x 16384 operands in seconds, so outputs are SAMPLED: every dX / dW entry depends
 on one row of each quantised operand, and the oracle quantises exactly those rows (their SR draws are keyed on the
@@ -21,18 +21,23 @@ def _bits(t):
     return t.contiguous().view(torch.int16).cpu().numpy().view(np.uint16)
 
 
-@pytest.mark.parametrize("layer_name", ["attn_out", "fc1"])
-def test_sampled_parity_at_6p7b_shapes(ref, layer_name):
+CASES = [("gpt_6p7b", "attn_out"), ("gpt_6p7b", "fc1"), ("gpt_6p7b", "qkv"), ("gpt_6p7b", "fc2"),
+         ("gpt_1p3b", "qkv"), ("gpt_1p3b", "attn_out"), ("gpt_1p3b", "fc1"), ("gpt_1p3b", "fc2"),
+         ("gpt_345m", "qkv"), ("gpt_345m", "attn_out"), ("gpt_345m", "fc1"), ("gpt_345m", "fc2")]
+
+
+@pytest.mark.parametrize("config,layer_name", CASES)
+def test_sampled_parity_at_full_shapes(ref, config, layer_name):
     import torch
     if not torch.cuda.is_available():
         pytest.skip("no GPU")
     from paper_2502_20586_b200 import binding as mx
 
-    layers, g = wl.CONFIGS["gpt_6p7b"]
+    layers, g = wl.CONFIGS[config]
     layer = [l for l in layers if l.name == layer_name][0]
     b, n, m = layer.b, layer.n, layer.m
     seed = 3
-    dY, X, W = wl.layer_inputs_device("gpt_6p7b", layer, seed=0)
+    dY, X, W = wl.layer_inputs_device(config, layer, seed=0)
     rng = np.random.default_rng(17)
     I = np.sort(rng.choice(b, 12, replace=False)); J = np.sort(rng.choice(n, 10, replace=False))       # dX[I, J]
     P = np.sort(rng.choice(m, 12, replace=False)); Q = np.sort(rng.choice(n, 10, replace=False))       # dW[P, Q]
