@@ -54,7 +54,8 @@ def _inputs(kind, shape, seed):
 # ------------------------------------------------------------------------------------------- quantiser
 
 @pytest.mark.parametrize("rounding", [0, 1])
-@pytest.mark.parametrize("reduce_dim,shape", [(1, (200, 1184)), (1, (3, 32)), (0, (544, 200)), (0, (32, 8))])
+@pytest.mark.parametrize("reduce_dim,shape", [(1, (200, 1184)), (1, (3, 32)), (0, (544, 200)), (0, (32, 8)),
+                                              (1, (200, 1280)), (0, (640, 200))])   # the last two: reduce length a multiple of 128
 def test_quantizer_bit_exact_without_rht(gpu, ref, rounding, reduce_dim, shape):
     """g = 0: both sides quantise the same fp32 values (the bf16 inputs), so everything is bit-exact.
     Shapes span several tiles and a ragged tail in both dimensions."""
