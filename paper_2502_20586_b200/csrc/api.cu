@@ -121,7 +121,7 @@ mxfp4_status make_codes_map(CUtensorMap* map, const uint8_t* codes, int64_t rows
 void attach_input_map(QuantArgs& a) {
     a.has_tmap = false;
     const int64_t K = a.reduce_dim == 1 ? a.cols : a.rows;
-    if (!(a.g == 32 || a.g == 64 || a.g == 128) || K % 128 != 0) return;
+    if (!(a.g == 32 || a.g == 64 || a.g == 128 || a.g == 256) || K % 128 != 0) return;
     if (a.rows > 0x7FFFFFFF || a.cols > 0x7FFFFFFF) return;
     const cuuint64_t dims[2] = {(cuuint64_t)a.cols, (cuuint64_t)a.rows};
     const cuuint64_t strides[1] = {(cuuint64_t)a.ld * 2};

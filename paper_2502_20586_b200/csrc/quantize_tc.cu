@@ -1,4 +1,4 @@
-// Blockwise RHT + MXFP4 quantiser with the transform on the tensor cores (g in {32, 64, 128}).
+// Blockwise RHT + MXFP4 quantiser with the transform on the tensor cores (g in {32, 64, 128, 256}).
 //
 // Section 3.2 builds the blockwise RHT as a dense matrix product with a small g x g matrix, which keeps it
 // memory-bound in the operand.  Here that product is a tcgen05.mma kind::f16: per tile of 128 output rows x 128
@@ -10,6 +10,10 @@
 // both access patterns: for a contiguous reduce dimension the x tile is the K-major A operand; for the transposing
 // views (W, dY^T, X^T of Algorithm 3) the very same TMA tile is handed to the MMA as an MN-major operand, so the
 // transposition costs nothing.
+//
+// g = 256 spans two 128-wide k-tiles: H_256 = [[H_128, H_128], [H_128, -H_128]], so the two k-tiles of a 256-chunk
+// go through their own half-transform T_h = diag(S_{128h..128h+127}) H_128 / 16 into two accumulators u and v, and
+// the epilogue forms u + v and u - v in fp32 (one add per element more than g <= 128).
 //
 // One launch can quantise up to four operand views that share g, seed and rounding (the four views of one
 // backward call, Algorithm 3 lines 3-6): their tiles form one list that the persistent CTAs walk, which removes
@@ -34,7 +38,7 @@ constexpr int kStagesQ = 4;
 constexpr uint32_t kBoxBytes = 64 * 2 * 128;        // one TMA box: 64 bf16 columns x 128 rows = 16 KB
 constexpr uint32_t kTileBytes = 2 * kBoxBytes;      // 32 KB
 constexpr uint32_t kTBytes = 2 * kBoxBytes;         // transform matrix, 128 x 128 bf16
-constexpr uint32_t kSmemQ = kStagesQ * kTileBytes + kTBytes + 1024 + 256;
+constexpr uint32_t kSmemQ = kStagesQ * kTileBytes + 2 * kTBytes + 1024 + 256;   // two transform matrices for g = 256
 constexpr int kAccBufs = 4;                         // 4 x 128 TMEM columns
 constexpr int kEpiGroups = 4;                       // epilogue warp groups (one warp per TMEM lane quadrant), on alternate tiles
 constexpr int kEpiWarps = 4 * kEpiGroups;
@@ -69,6 +73,13 @@ struct QMaps {
 };
 
 // bf16 entry (n, k) of the transform operand, stored N x K (K-major): T[k][n] = S_k H_g[k][n] inside a g-chunk.
+// g = 256 (Sylvester: H_256 = [[H_128, H_128], [H_128, -H_128]]): entry (n, k) of the half-transform h, T_h[k][n] =
+// S_{128 h + k} H_128[k][n] / 16; the epilogue combines u = A_lo T_0 and v = A_hi T_1 into u + v and u - v.
+__device__ __forceinline__ uint32_t transform_entry_256(int n, int k, const uint32_t (&sign)[4]) {
+    const uint32_t neg = ((sign[k >> 5] >> (k & 31)) ^ (uint32_t)__popc(k & n)) & 1u;
+    return 0x3D80u | (neg << 15);                                         // 1/16 = exact 1/sqrt(256)
+}
+
 __device__ __forceinline__ uint32_t transform_entry(int n, int k, int g, const uint32_t (&sign)[4]) {
     if ((n ^ k) & ~(g - 1)) return 0u;                                   // different g-chunks
     const int kk = k & (g - 1);
@@ -113,13 +124,14 @@ __device__ __forceinline__ TilePos advance_tile(const QParams& p, const TilePos&
 
 enum { kModeSR = 0, kModeRN = 1, kModeDump = 2 };
 
-template <int MODE>
+// KW = 128-wide k-tiles per entry of the tile list: 1, or 2 for g = 256 (a tile then spans one 256-chunk).
+template <int MODE, int KW>
 __global__ void __launch_bounds__(kThreadsQ, 1)
 quantize_tc_kernel(const __grid_constant__ QMaps maps, const __grid_constant__ QParams p) {
     extern __shared__ uint8_t smem_raw[];
     uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
     uint8_t* smem_t = smem + kStagesQ * kTileBytes;
-    uint64_t* bars = reinterpret_cast<uint64_t*>(smem_t + kTBytes);
+    uint64_t* bars = reinterpret_cast<uint64_t*>(smem_t + 2 * kTBytes);
     uint64_t* full_bar = bars;                          // [kStagesQ]  TMA -> MMA
     uint64_t* empty_bar = bars + kStagesQ;              // [kStagesQ]  MMA -> TMA
     uint64_t* acc_full = bars + 2 * kStagesQ;           // [kAccBufs]  MMA -> epilogue
@@ -132,7 +144,7 @@ quantize_tc_kernel(const __grid_constant__ QMaps maps, const __grid_constant__ Q
 
     if (threadIdx.x == 0) {
         for (int s = 0; s < kStagesQ; ++s) { mbar_init(&full_bar[s], 1); mbar_init(&empty_bar[s], 1); }
-        for (int b = 0; b < kAccBufs; ++b) { mbar_init(&acc_full[b], 1); mbar_init(&acc_empty[b], 4); }
+        for (int b = 0; b < kAccBufs; ++b) { mbar_init(&acc_full[b], 1); mbar_init(&acc_empty[b], KW == 2 ? 8 : 4); }
         *abort_flag = 0;
         mbar_fence_init();
         for (int v = 0; v < p.n_views; ++v) prefetch_tensormap(&maps.x[v]);
@@ -144,16 +156,22 @@ quantize_tc_kernel(const __grid_constant__ QMaps maps, const __grid_constant__ Q
     {
         // Transform operand, written in the 128-byte-swizzled K-major layout the MMA descriptor expects:
         // entry (n, k) at box (k / 64), row n (128 B pitch), 16-byte chunk ((k % 64) / 8) ^ (n % 8).
-        const uint4 o = philox4x32_10(0u, 0u, 0u, 0u, (uint32_t)p.seed, (uint32_t)(p.seed >> 32));
-        const uint32_t sign[4] = {o.x, o.y, o.z, o.w};
-        for (int task = threadIdx.x; task < 128 * 16; task += kThreadsQ) {
-            const int n = task >> 4, c = task & 15;                      // c: 16-byte chunk = 8 consecutive k
-            uint32_t w[4];
 #pragma unroll
-            for (int j = 0; j < 4; ++j)
-                w[j] = transform_entry(n, c * 8 + 2 * j, p.g, sign) | (transform_entry(n, c * 8 + 2 * j + 1, p.g, sign) << 16);
-            const uint32_t off = (uint32_t)(c >> 3) * kBoxBytes + (uint32_t)n * 128u + (uint32_t)(((c & 7) ^ (n & 7)) << 4);
-            *reinterpret_cast<uint4*>(smem_t + off) = make_uint4(w[0], w[1], w[2], w[3]);
+        for (int h = 0; h < KW; ++h) {                                   // KW = 2: sign bits 128 h .. 128 h + 127 come from Philox call h
+            const uint4 o = philox4x32_10((uint32_t)h, 0u, 0u, 0u, (uint32_t)p.seed, (uint32_t)(p.seed >> 32));
+            const uint32_t sign[4] = {o.x, o.y, o.z, o.w};
+            for (int task = threadIdx.x; task < 128 * 16; task += kThreadsQ) {
+                const int n = task >> 4, c = task & 15;                  // c: 16-byte chunk = 8 consecutive k
+                uint32_t w[4];
+#pragma unroll
+                for (int j = 0; j < 4; ++j) {
+                    const int k0 = c * 8 + 2 * j;
+                    w[j] = KW == 2 ? (transform_entry_256(n, k0, sign) | (transform_entry_256(n, k0 + 1, sign) << 16))
+                                   : (transform_entry(n, k0, p.g, sign) | (transform_entry(n, k0 + 1, p.g, sign) << 16));
+                }
+                const uint32_t off = (uint32_t)(c >> 3) * kBoxBytes + (uint32_t)n * 128u + (uint32_t)(((c & 7) ^ (n & 7)) << 4);
+                *reinterpret_cast<uint4*>(smem_t + h * kTBytes + off) = make_uint4(w[0], w[1], w[2], w[3]);
+            }
         }
         fence_proxy_async_smem();                                        // generic-proxy writes -> tensor-core reads
     }
@@ -167,17 +185,21 @@ quantize_tc_kernel(const __grid_constant__ QMaps maps, const __grid_constant__ Q
         if (lane == 0) {
             uint32_t it = 0;
             bool ok = true;
-            for (uint32_t t = blockIdx.x; t < num_tiles; t += gridDim.x, ++it) {
-                const int s = it % kStagesQ;
-                if (!(ok = mbar_wait(&empty_bar[s], ((it / kStagesQ) & 1) ^ 1, abort_flag))) break;
+            for (uint32_t t = blockIdx.x; t < num_tiles && ok; t += gridDim.x) {
                 const TilePos pos = locate_tile(p, t);
                 // x coordinates: (column, row).  reduce_dim 1: output rows = x rows, k = x columns; else swapped.
                 const bool rowwise = p.view[pos.v].reduce_dim == 1;
-                const int32_t cx = (int32_t)((rowwise ? pos.kt : pos.rt) * kTile), cy = (int32_t)((rowwise ? pos.rt : pos.kt) * kTile);
-                uint8_t* st = smem + s * kTileBytes;
-                mbar_expect_tx(&full_bar[s], kTileBytes);
-                tma_load_2d(st, &maps.x[pos.v], &full_bar[s], cx, cy);
-                tma_load_2d(st + kBoxBytes, &maps.x[pos.v], &full_bar[s], cx + 64, cy);
+#pragma unroll
+                for (int h = 0; h < KW; ++h, ++it) {
+                    const int s = it % kStagesQ;
+                    if (!(ok = mbar_wait(&empty_bar[s], ((it / kStagesQ) & 1) ^ 1, abort_flag))) break;
+                    const uint32_t kt = pos.kt * KW + h;                 // 128-wide k-tile
+                    const int32_t cx = (int32_t)((rowwise ? kt : pos.rt) * kTile), cy = (int32_t)((rowwise ? pos.rt : kt) * kTile);
+                    uint8_t* st = smem + s * kTileBytes;
+                    mbar_expect_tx(&full_bar[s], kTileBytes);
+                    tma_load_2d(st, &maps.x[pos.v], &full_bar[s], cx, cy);
+                    tma_load_2d(st + kBoxBytes, &maps.x[pos.v], &full_bar[s], cx + 64, cy);
+                }
             }
             if (!ok) *abort_flag = 1;
         }
@@ -190,30 +212,33 @@ quantize_tc_kernel(const __grid_constant__ QMaps maps, const __grid_constant__ Q
             const uint32_t t_addr = smem_u32(smem_t);
             uint32_t it = 0;
             bool ok = true;
-            for (uint32_t t = blockIdx.x; t < num_tiles; t += gridDim.x, ++it) {
-                const int s = it % kStagesQ, b = it % kAccBufs;
+            for (uint32_t t = blockIdx.x; t < num_tiles && ok; t += gridDim.x) {
                 int v = 0;
 #pragma unroll
                 for (int i = 1; i < kQuantMaxViews; ++i)
                     if (i < p.n_views && t >= p.view[i].tile_begin) v = i;
                 const bool rowwise = p.view[v].reduce_dim == 1;
                 const uint32_t idesc = idesc_k | ((rowwise ? 0u : 1u) << 15);
-                if (!(ok = mbar_wait(&acc_empty[b], ((it / kAccBufs) & 1) ^ 1, abort_flag))) break;
-                if (!(ok = mbar_wait(&full_bar[s], (it / kStagesQ) & 1, abort_flag))) break;
-                tc_fence_after_sync();
-                const uint32_t a_addr = smem_u32(smem + s * kTileBytes);
 #pragma unroll
-                for (int ks = 0; ks < 8; ++ks) {                           // K = 16 per MMA
-                    uint64_t adesc;
-                    if (rowwise)                // K-major: box ks/4, 32 bytes of K per step inside the 128-byte swizzle atom
-                        adesc = make_smem_desc(a_addr + (ks >> 2) * kBoxBytes + (ks & 3) * 32, 16, 1024, 2);
-                    else                        // MN-major: 16 k-rows of 128 B per step; the second 64 output rows sit one box further
-                        adesc = make_smem_desc(a_addr + ks * 2048, kBoxBytes, 1024, 2);
-                    const uint64_t bdesc = make_smem_desc(t_addr + (ks >> 2) * kBoxBytes + (ks & 3) * 32, 16, 1024, 2);
-                    tc_mma_f16(tmem_base + b * kTile, adesc, bdesc, idesc, ks != 0 ? 1u : 0u);
+                for (int h = 0; h < KW; ++h, ++it) {                       // KW = 2: k-tile h goes through T_h into its own accumulator
+                    const int s = it % kStagesQ, b = it % kAccBufs;
+                    if (!(ok = mbar_wait(&acc_empty[b], ((it / kAccBufs) & 1) ^ 1, abort_flag))) break;
+                    if (!(ok = mbar_wait(&full_bar[s], (it / kStagesQ) & 1, abort_flag))) break;
+                    tc_fence_after_sync();
+                    const uint32_t a_addr = smem_u32(smem + s * kTileBytes);
+#pragma unroll
+                    for (int ks = 0; ks < 8; ++ks) {                       // K = 16 per MMA
+                        uint64_t adesc;
+                        if (rowwise)            // K-major: box ks/4, 32 bytes of K per step inside the 128-byte swizzle atom
+                            adesc = make_smem_desc(a_addr + (ks >> 2) * kBoxBytes + (ks & 3) * 32, 16, 1024, 2);
+                        else                    // MN-major: 16 k-rows of 128 B per step; the second 64 output rows sit one box further
+                            adesc = make_smem_desc(a_addr + ks * 2048, kBoxBytes, 1024, 2);
+                        const uint64_t bdesc = make_smem_desc(t_addr + h * kTBytes + (ks >> 2) * kBoxBytes + (ks & 3) * 32, 16, 1024, 2);
+                        tc_mma_f16(tmem_base + b * kTile, adesc, bdesc, idesc, ks != 0 ? 1u : 0u);
+                    }
+                    tc_commit(&empty_bar[s]);
+                    tc_commit(&acc_full[b]);
                 }
-                tc_commit(&empty_bar[s]);
-                tc_commit(&acc_full[b]);
             }
             if (!ok) *abort_flag = 1;
         }
@@ -232,7 +257,7 @@ quantize_tc_kernel(const __grid_constant__ QMaps maps, const __grid_constant__ Q
         bool ok = true;
 
         auto first_elem = [&](const TilePos& pos) -> uint64_t {          // linear index of this thread's first element
-            return (uint64_t)(pos.rt * (uint32_t)kTile + lane_row) * (uint64_t)p.view[pos.v].K + (uint64_t)(pos.kt * (uint32_t)kTile);
+            return (uint64_t)(pos.rt * (uint32_t)kTile + lane_row) * (uint64_t)p.view[pos.v].K + (uint64_t)(pos.kt * (uint32_t)(kTile * KW));
         };
 
         uint32_t it = (uint32_t)grp;
@@ -240,6 +265,84 @@ quantize_tc_kernel(const __grid_constant__ QMaps maps, const __grid_constant__ Q
         TilePos pos = locate_tile(p, t < num_tiles ? t : 0u);
         uint32_t rw[8];
         if (MODE == kModeSR) sr_draws32(p.keys, p.view[pos.v].stream_tag, first_elem(pos), rw);
+        if (KW == 2) {
+            // g = 256: a tile is one 256-chunk of 128 rows; its two k-tiles went through T_0 and T_1 into the accumulator
+            // pair (b0, b0 + 1): u = A_lo T_0, v = A_hi T_1.  The transformed values are y[0..127] = u + v and
+            // y[128..255] = u - v (H_256 = [[H, H], [H, -H]]).  Tiles alternate between the two accumulator pairs; pair
+            // pr is drained by groups 2 pr (the u + v half) and 2 pr + 1 (the u - v half), so every barrier is used by
+            // the same warps each time and its phases alternate for them.
+            const int pr = grp >> 1, hh = grp & 1;
+            const uint32_t stride2 = 2u * gridDim.x;
+            it = (uint32_t)pr;
+            t = blockIdx.x + it * gridDim.x;
+            pos = locate_tile(p, t < num_tiles ? t : 0u);
+            if (MODE == kModeSR) sr_draws32(p.keys, p.view[pos.v].stream_tag, first_elem(pos) + 128u * hh, rw);
+            for (; t < num_tiles; t += stride2, it += 2) {
+                const int b0 = 2 * pr;
+                const QView& vw = p.view[pos.v];
+                const uint32_t rt = pos.rt, kt = pos.kt;
+                const int64_t K = vw.K;
+                const int64_t row = (int64_t)rt * kTile + lane_row;
+                const int64_t k0 = (int64_t)kt * (2 * kTile) + 128 * hh;        // this group's 128 elements of the row
+                const bool live = row < vw.R;
+                uint8_t* code_dst = vw.codes + row * (K >> 1) + (k0 >> 1);
+                const uint32_t nkb = (uint32_t)(K >> 5), nkc = (nkb + 3) >> 2;
+                uint8_t* scale_dst = vw.scales + (p.sf_native ? ((int64_t)(rt * nkc + 2 * kt + hh) * 512 + lane * 16 + q * 4) : row * nkb + (k0 >> 5));
+                float* y_dst = MODE == kModeDump ? vw.y_out + row * K + k0 : nullptr;
+                const uint64_t i_cur = first_elem(pos) + 128u * hh;
+                const uint32_t tag_cur = vw.stream_tag;
+                pos = t + stride2 < num_tiles ? advance_tile(p, pos, t + stride2) : locate_tile(p, 0u);
+                const uint64_t i_next = first_elem(pos) + 128u * hh;
+                const uint32_t tag_next = p.view[pos.v].stream_tag;
+                const uint32_t ph = (it >> 1) & 1;                               // this pair's (it / 2)-th use
+                ok = mbar_wait(&acc_full[b0], ph, abort_flag) && mbar_wait(&acc_full[b0 + 1], ph, abort_flag);
+                ok = __all_sync(0xffffffffu, ok);
+                if (!ok) break;
+                tc_fence_after_sync();
+                const uint32_t ta = tmem_base + ((uint32_t)(q * 32) << 16) + b0 * kTile;
+                uint32_t sb_all = 0;
+#pragma unroll
+                for (int j = 0; j < 4; ++j) {
+                    uint32_t nx[8], packed[4], sb = 0;
+                    float y[32];
+#pragma unroll
+                    for (int c = 0; c < 2; ++c) {                           // sixteen columns of u and of v at a time
+                        uint32_t u[16], v[16];
+                        tmem_ld_32x32b_x16(ta + 32 * j + 16 * c, u);
+                        tmem_ld_32x32b_x16(ta + kTile + 32 * j + 16 * c, v);
+                        tmem_ld_wait();
+#pragma unroll
+                        for (int i = 0; i < 16; ++i)
+                            y[16 * c + i] = hh == 0 ? __uint_as_float(u[i]) + __uint_as_float(v[i]) : __uint_as_float(u[i]) - __uint_as_float(v[i]);
+                    }
+                    if (j == 3) {                                           // this group is done with both accumulators
+                        tc_fence_before_sync();
+                        __syncwarp();
+                        if (lane == 0) { mbar_arrive(&acc_empty[b0]); mbar_arrive(&acc_empty[b0 + 1]); }
+                    }
+                    if (MODE == kModeSR) {
+                        if (j < 3) sr_draws32(p.keys, tag_cur, i_cur + 32 * (j + 1), nx);
+                        else sr_draws32(p.keys, tag_next, i_next, nx);
+                    }
+                    if (MODE == kModeDump) {
+                        if (live) {
+                            float4* dst = reinterpret_cast<float4*>(y_dst + 32 * j);
+#pragma unroll
+                            for (int i = 0; i < 8; ++i) dst[i] = make_float4(y[4 * i], y[4 * i + 1], y[4 * i + 2], y[4 * i + 3]);
+                        }
+                    } else {
+                        quantize_block32_rw<MODE>(y, rw, packed, sb, p.pipe);
+                        if (live) *reinterpret_cast<uint4*>(code_dst + 16 * j) = make_uint4(packed[0], packed[1], packed[2], packed[3]);
+                        sb_all |= sb << (8 * j);
+                    }
+                    if (MODE == kModeSR) {
+#pragma unroll
+                        for (int i = 0; i < 8; ++i) rw[i] = nx[i];
+                    }
+                }
+                if (MODE != kModeDump && live) *reinterpret_cast<uint32_t*>(scale_dst) = sb_all;
+            }
+        } else
         for (; t < num_tiles; t += stride, it += kEpiGroups) {
             const int b = it % kAccBufs;
             const QView& vw = p.view[pos.v];
@@ -321,15 +424,18 @@ bool quant_tc_eligible(const QuantArgs& a) {
     const int64_t K = a.reduce_dim == 1 ? a.cols : a.rows;
     const int64_t R = a.reduce_dim == 1 ? a.rows : a.cols;
     const int64_t tiles = ((R + kTile - 1) / kTile) * (K / kTile);          // tile indices are 32-bit in the kernel
-    return (a.g == 32 || a.g == 64 || a.g == 128) && K % kTile == 0 && tiles < (int64_t(1) << 28) && a.has_tmap;
+    return (a.g == 32 || a.g == 64 || a.g == 128 || a.g == 256) && K % kTile == 0 && tiles < (int64_t(1) << 28) && a.has_tmap;
 }
 
 cudaError_t quant_tc_init() {
-    cudaError_t e = cudaFuncSetAttribute(quantize_tc_kernel<kModeSR>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kSmemQ);
-    if (e != cudaSuccess) return e;
-    e = cudaFuncSetAttribute(quantize_tc_kernel<kModeRN>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kSmemQ);
-    if (e != cudaSuccess) return e;
-    return cudaFuncSetAttribute(quantize_tc_kernel<kModeDump>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kSmemQ);
+    const void* kernels[6] = {(const void*)quantize_tc_kernel<kModeSR, 1>, (const void*)quantize_tc_kernel<kModeRN, 1>,
+                              (const void*)quantize_tc_kernel<kModeDump, 1>, (const void*)quantize_tc_kernel<kModeSR, 2>,
+                              (const void*)quantize_tc_kernel<kModeRN, 2>, (const void*)quantize_tc_kernel<kModeDump, 2>};
+    for (const void* k : kernels) {
+        const cudaError_t e = cudaFuncSetAttribute(k, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kSmemQ);
+        if (e != cudaSuccess) return e;
+    }
+    return cudaSuccess;
 }
 
 // Quantise n (1..kQuantMaxViews) eligible operand views that share g, seed, rounding and scale layout in one launch.
@@ -343,7 +449,7 @@ cudaError_t launch_quantize_tc_group(const QuantArgs* a, int n, bool dump_y, cud
         w.R = a[v].reduce_dim == 1 ? a[v].rows : a[v].cols;
         w.K = a[v].reduce_dim == 1 ? a[v].cols : a[v].rows;
         w.r_tiles = (uint32_t)((w.R + kTile - 1) / kTile);
-        w.k_tiles = (uint32_t)(w.K / kTile);
+        w.k_tiles = (uint32_t)(w.K / (a[v].g == 256 ? 2 * kTile : kTile));     // g = 256: a tile spans one 256-chunk
         w.tile_begin = tiles;
         w.n_tiles = w.r_tiles * w.k_tiles;
         tiles += w.n_tiles;
@@ -373,15 +479,21 @@ cudaError_t launch_quantize_tc_group(const QuantArgs* a, int n, bool dump_y, cud
     for (int v = 0; v < kQuantMaxViews; ++v) {              // the two epilogue groups step through the list by 2 * grid
         QView& w = p.view[v];
         w.minor_count = w.reduce_dim == 1 ? w.k_tiles : w.r_tiles;
-        w.d_major = (uint32_t)kEpiGroups * grid / w.minor_count;
-        w.d_minor = (uint32_t)kEpiGroups * grid % w.minor_count;
+        const uint32_t step = (p.g == 256 ? 2u : (uint32_t)kEpiGroups) * grid;   // g = 256: the groups work in pairs
+        w.d_major = step / w.minor_count;
+        w.d_minor = step % w.minor_count;
     }
-    if (dump_y)
-        quantize_tc_kernel<kModeDump><<<grid, kThreadsQ, kSmemQ, stream>>>(maps, p);
-    else if (a[0].rounding == 0)
-        quantize_tc_kernel<kModeSR><<<grid, kThreadsQ, kSmemQ, stream>>>(maps, p);
-    else
-        quantize_tc_kernel<kModeRN><<<grid, kThreadsQ, kSmemQ, stream>>>(maps, p);
+    const bool wide = p.g == 256;
+    if (dump_y) {
+        if (wide) quantize_tc_kernel<kModeDump, 2><<<grid, kThreadsQ, kSmemQ, stream>>>(maps, p);
+        else quantize_tc_kernel<kModeDump, 1><<<grid, kThreadsQ, kSmemQ, stream>>>(maps, p);
+    } else if (a[0].rounding == 0) {
+        if (wide) quantize_tc_kernel<kModeSR, 2><<<grid, kThreadsQ, kSmemQ, stream>>>(maps, p);
+        else quantize_tc_kernel<kModeSR, 1><<<grid, kThreadsQ, kSmemQ, stream>>>(maps, p);
+    } else {
+        if (wide) quantize_tc_kernel<kModeRN, 2><<<grid, kThreadsQ, kSmemQ, stream>>>(maps, p);
+        else quantize_tc_kernel<kModeRN, 1><<<grid, kThreadsQ, kSmemQ, stream>>>(maps, p);
+    }
     return cudaGetLastError();
 }
 
