@@ -141,6 +141,10 @@ def mxfp4_linear_backward(dY, X, W, g: int, seed: int, rounding: int = ROUND_SR,
     return dX, dW
 
 
+def mxfp4_linear_backward_ex_workspace(b: int, m: int, n: int, with_bias: bool) -> int:
+    return int(_lib.mxfp4_linear_backward_ex_workspace(b, m, n, 1 if with_bias else 0))
+
+
 def mxfp4_linear_backward_ex(dY, X, W, g: int, seed: int, rounding: int = ROUND_SR, out_dtype: int = OUT_BF16,
                              dX=None, dW=None, db=None, with_bias: bool = False, accumulate: bool = False, workspace=None):
     """Algorithm 3 plus the bias gradient (fp32 [m], column sums of dY) and accumulation into fp32 dW / db.
@@ -158,7 +162,7 @@ def mxfp4_linear_backward_ex(dY, X, W, g: int, seed: int, rounding: int = ROUND_
     if db is None and with_bias:
         assert not accumulate, "accumulation needs an existing db"
         db = torch.empty((m,), dtype=torch.float32, device=dY.device)
-    need = int(_lib.mxfp4_linear_backward_ex_workspace(b, m, n, 1 if db is not None else 0))
+    need = mxfp4_linear_backward_ex_workspace(b, m, n, db is not None)
     if workspace is None:
         workspace = torch.empty(need, dtype=torch.uint8, device=dY.device)
     _check(_lib.mxfp4_linear_backward_ex(_ptr(dY), _ptr(X), _ptr(W), b, m, n, g, rounding, seed, _ptr(dX), _ptr(dW),

@@ -84,7 +84,7 @@ def main(argv=None):
         dW = torch.zeros((m, n), dtype=dt, device=dev)
         if args.bias or args.accumulate:
             db = torch.zeros((m,), dtype=torch.float32, device=dev) if args.bias else None
-            ws = torch.empty(mx.mxfp4_linear_backward_workspace(b, m, n) + (64 * m * 4 + 1024), dtype=torch.uint8, device=dev)
+            ws = torch.empty(mx.mxfp4_linear_backward_ex_workspace(b, m, n, args.bias), dtype=torch.uint8, device=dev)
             fn = lambda: mx.mxfp4_linear_backward_ex(dY, X, W, g, 0, args.rounding, out_dtype, dX=dX, dW=dW, db=db,
                                                      accumulate=args.accumulate, workspace=ws)
         else:
