@@ -287,3 +287,29 @@ def test_bias_grad_and_accumulation(gpu, ref, b, m, n):
     with pytest.raises(gpu.MxFp4Error):
         gpu.mxfp4_linear_backward_ex(_dev(dY), _dev(X), _dev(W), 64, 5, gpu.ROUND_SR, gpu.OUT_BF16,
                                      dW=torch.zeros((m, n), dtype=torch.bfloat16, device="cuda"), accumulate=True)
+
+
+def test_linear_backward_captures_into_a_cuda_graph(gpu):
+    """A shape large enough for the fork / join of the two GEMMs: the captured graph replays to the same bits."""
+    import torch
+    gen = torch.Generator(device="cuda").manual_seed(1)
+    b, n, m, g = 4096, 2048, 4096, 128
+    dY = (torch.randn((b, m), generator=gen, device="cuda") * 1e-3).to(torch.bfloat16)
+    X = torch.randn((b, n), generator=gen, device="cuda").to(torch.bfloat16)
+    W = (torch.randn((m, n), generator=gen, device="cuda") * 0.02).to(torch.bfloat16)
+    dX = torch.empty((b, n), dtype=torch.bfloat16, device="cuda")
+    dW = torch.empty((m, n), dtype=torch.bfloat16, device="cuda")
+    ws = torch.empty(gpu.mxfp4_linear_backward_workspace(b, m, n), dtype=torch.uint8, device="cuda")
+    gpu.mxfp4_linear_backward(dY, X, W, g, 7, gpu.ROUND_SR, gpu.OUT_BF16, dX=dX, dW=dW, workspace=ws)
+    torch.cuda.synchronize()
+    want_x, want_w = dX.clone(), dW.clone()
+    dX.zero_(); dW.zero_()
+    graph = torch.cuda.CUDAGraph()
+    side = torch.cuda.Stream()
+    with torch.cuda.stream(side):
+        with torch.cuda.graph(graph, stream=side):
+            gpu.mxfp4_linear_backward(dY, X, W, g, 7, gpu.ROUND_SR, gpu.OUT_BF16, dX=dX, dW=dW, workspace=ws)
+    graph.replay()
+    torch.cuda.synchronize()
+    assert torch.equal(dX, want_x) and torch.equal(dW, want_w)
+    assert gpu.mxfp4_device_status() == 0
