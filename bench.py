@@ -106,21 +106,21 @@ class ClockSampler:
 
 
 # ------------------------------------------------------------------------------------------ reference arm
-def oracle_sample(config: str, seed: int = 0):
-    """A bounded sample of the workload for the CPU oracle: Algorithm 3 on a 4096-token slab of the
-    attention-output layer, dX in full and dW on up to 4096 sampled rows.  Returns (fn, flops, description)."""
+def oracle_sample(config: str, seed: int = 0, tokens: int = 4096, dw_sample: int = 4096):
+    """A bounded sample of the workload for the CPU oracle: Algorithm 3 on a `tokens`-token slab of the
+    attention-output layer, dX in full and dW on up to `dw_sample` sampled rows.  Returns (fn, flops, description, threads)."""
     import numpy as np
     from oracle import ref
     from paper_2502_20586_b200 import workloads as wl
     layers, g = wl.CONFIGS[config]
     layer = [l for l in layers if l.name in ("attn_out", "single")][0]
-    b_s = min(4096, layer.b)
+    b_s = min(tokens, layer.b)
     rng = np.random.default_rng(seed)
     std = 1e-3 if config == "single_256x512" else 1e-4
     dY = wl.grad_like(rng, (b_s, layer.m), std)
     X = wl.activation_like(rng, (b_s, layer.n), n_outlier_channels=8)
     W = wl.weight_like(rng, (layer.m, layer.n))
-    dw_rows = np.sort(rng.choice(layer.m, size=min(4096, layer.m), replace=False))
+    dw_rows = np.sort(rng.choice(layer.m, size=min(dw_sample, layer.m), replace=False))
     flops = 2 * b_s * layer.n * layer.m + 2 * len(dw_rows) * layer.n * b_s
 
     def run():
@@ -135,7 +135,8 @@ def run_reference(args):
     rank = int(os.environ.get("RANK", "0"))
     if rank != 0:
         return
-    run, flops, desc, cores = oracle_sample(args.config)
+    # each step is a quarter of the cpu_baseline sample (about 2 s), so that 40 steps still end within two minutes
+    run, flops, desc, cores = oracle_sample(args.config, tokens=2048, dw_sample=2048)
     for _ in range(min(args.warmup, 1)):
         run()
     t0 = time.perf_counter()
