@@ -28,16 +28,17 @@ __device__ __forceinline__ void unpack_bf16x8(const uint4& q, float* v) {
 // v <- v diag(S) H_g / sqrt(g) for the 32 values of this thread; lanes [lane & ~(G/32-1) ...) share a chunk.
 template <int G>
 __device__ __forceinline__ void rht_in_place(float (&v)[32], uint32_t sign_bits, int lane, int lane_stride) {
-    if (G == 0) return;
+    if constexpr (G != 0) {
 #pragma unroll
-    for (int i = 0; i < 32; ++i) v[i] = (sign_bits >> i) & 1u ? -v[i] : v[i];
-    fwht32(v);
-    if (G >= 64) fwht_cross(v, lane_stride, lane);
-    if (G >= 128) fwht_cross(v, lane_stride * 2, lane);
-    if (G >= 256) fwht_cross(v, lane_stride * 4, lane);
-    const float c = inv_sqrt_g(G);
+        for (int i = 0; i < 32; ++i) v[i] = (sign_bits >> i) & 1u ? -v[i] : v[i];
+        fwht32(v);
+        if (G >= 64) fwht_cross(v, lane_stride, lane);
+        if (G >= 128) fwht_cross(v, lane_stride * 2, lane);
+        if (G >= 256) fwht_cross(v, lane_stride * 4, lane);
+        const float c = inv_sqrt_g(G);
 #pragma unroll
-    for (int i = 0; i < 32; ++i) v[i] *= c;
+        for (int i = 0; i < 32; ++i) v[i] *= c;
+    }
 }
 
 // ------------------------------------------------------------------------------------------------ rowwise
