@@ -78,6 +78,21 @@ def test_argument_validation_needs_no_device(lib):
     assert lb(P, P, P, 256, 512, 512, 64, 0, 0, P, P, 0, 0, 1 << 30, 0) == 6      # workspace NULL
     assert lb(P, P, P, 256, 512, 512, 64, 0, 0, P, P, 0, P, 1024, 0) == 6         # too small
     assert lb(P, P, P, 256, 512, 512, 64, 0, 0, P, P, 0, P + 16, 1 << 30, 0) == 6  # misaligned
+    # extended form: bias gradient and accumulation
+    ex = raw.mxfp4_linear_backward_ex
+    big = 1 << 30
+    assert ex(P, P, P, 256, 512, 512, 64, 0, 0, P, 0, P, 1, 0, P, big, 0) == 1         # dW NULL
+    assert ex(P, P, P, 256, 512, 512, 64, 0, 0, P, P, P, 0, 1, P, big, 0) == 5         # accumulate needs fp32 outputs
+    assert ex(P, P, P, 256, 512, 512, 64, 0, 0, P, P, P, 1, 2, P, big, 0) == 5         # accumulate selector
+    assert ex(P, P, P, 256, 512, 512, 64, 0, 0, P, P, P + 4, 1, 0, P, big, 0) == 3     # db alignment
+    need0 = raw.mxfp4_linear_backward_ex_workspace(256, 512, 512, 0)
+    need1 = raw.mxfp4_linear_backward_ex_workspace(256, 512, 512, 1)
+    assert need0 == raw.mxfp4_linear_backward_workspace(256, 512, 512) and need1 > need0 and need1 % 256 == 0
+    assert ex(P, P, P, 256, 512, 512, 64, 0, 0, P, P, P, 1, 0, P, need0, 0) == 6       # the bias scratch is missing
+    assert raw.mxfp4_linear_backward_ex_workspace(256, 0, 512, 1) == 0
+    # measurement aid
+    assert raw.mxfp4_fp4_ceiling(0, C.byref(C.c_int64(0)), 0) == 2
+    assert raw.mxfp4_fp4_ceiling(64, None, 0) == 2
 
 
 def test_binding_fails_loudly_without_library(tmp_path, monkeypatch):
