@@ -243,6 +243,7 @@ gemm_mxf4_pair_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_c
         const int q = warp & 3;
         uint8_t* stage0 = epi_ring + q * 2 * kEpiBuf;
         uint32_t n_stores = 0;                                  // bulk groups this warp committed so far
+        const uint64_t pol_c = l2_policy_evict_first();         // the output is not read again here: let the operands keep L2
         bool ok = true;
         // One staged block: 16 registers = 64 bytes of this lane's row, columns [col, col + 64 B).
         auto put = [&](const uint32_t (&w)[16], int32_t col, int32_t row0, bool in_range) {
@@ -260,7 +261,7 @@ gemm_mxf4_pair_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_c
             if (lane == 0) {
                 if (in_range) {
                     if (p.accumulate) tma_reduce_add_2d(&tmap_c, buf, col, row0);
-                    else tma_store_2d(&tmap_c, buf, col, row0);
+                    else tma_store_2d_hint(&tmap_c, buf, col, row0, pol_c);
                 }
                 bulk_commit_group();
             }
