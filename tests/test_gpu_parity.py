@@ -313,3 +313,20 @@ def test_linear_backward_captures_into_a_cuda_graph(gpu):
     torch.cuda.synchronize()
     assert torch.equal(dX, want_x) and torch.equal(dW, want_w)
     assert gpu.mxfp4_device_status() == 0
+
+
+def test_linear_backward_is_bitwise_reproducible(gpu):
+    """Same inputs, same seed: the same bits, call after call (fixed MMA order, fixed summation order of the bias sums)."""
+    import torch
+    gen = torch.Generator(device="cuda").manual_seed(9)
+    b, n, m, g = 4096, 2048, 4096, 128
+    dY = (torch.randn((b, m), generator=gen, device="cuda") * 1e-3).to(torch.bfloat16)
+    X = torch.randn((b, n), generator=gen, device="cuda").to(torch.bfloat16)
+    W = (torch.randn((m, n), generator=gen, device="cuda") * 0.02).to(torch.bfloat16)
+    first = gpu.mxfp4_linear_backward_ex(dY, X, W, g, 21, gpu.ROUND_SR, gpu.OUT_FP32, with_bias=True)
+    for _ in range(3):
+        again = gpu.mxfp4_linear_backward_ex(dY, X, W, g, 21, gpu.ROUND_SR, gpu.OUT_FP32, with_bias=True)
+        assert all(torch.equal(a, c) for a, c in zip(first, again))
+    other = gpu.mxfp4_linear_backward_ex(dY, X, W, g, 22, gpu.ROUND_SR, gpu.OUT_FP32, with_bias=True)
+    assert not torch.equal(first[0], other[0]) and torch.equal(first[2], other[2])      # the seed moves dX, not the bias sums
+    assert gpu.mxfp4_device_status() == 0
