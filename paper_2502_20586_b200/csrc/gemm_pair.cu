@@ -4,16 +4,19 @@
 // 1-CTA kernel (gemm.cu) is bound by exactly that operand traffic.  Each CTA keeps the accumulator of its own 128
 // rows (all 256 columns) in its TMEM.
 //
-// The scale tiles travel in their own, deeper ring (8 slots, decoupled from the 6 operand stages), so they are in
-// TMEM long before the MMAs that need them; the only tight loop left is the reuse of an operand stage.
+// Shared memory (all 227 KB): six operand stages of 32 KB, a six-slot scale ring of 3 KB, 16 KB of epilogue staging.
+// TMEM: 256 accumulator columns + six scale slots of 24 columns.
 //
-// Roles per CTA (11 warps), all waits bounded as in gemm.cu:
-//   warp 0      TMA producer: own A rows, own half of B (completion counted on the LEADER's barrier);
-//   warp 10     scale loader: own A-row scale tiles and the scale tiles of all 256 B rows, bulk copies into the ring;
-//   warp 1      MMA issuer, leader CTA only: four K = 64 pair-MMAs per stage; tcgen05.commit frees stage, scale slot
-//               and accumulator in BOTH CTAs;
-//   warps 2..5  epilogue of the CTA's own 128 x 256 half tile;
-//   warps 6..9  scale movers: shared memory -> registers -> own TMEM (tcgen05.st), then arrive on the leader's barrier.
+// Roles per CTA (12 warps), all waits bounded as in gemm.cu:
+//   warp 0       TMA producer: own A rows, own half of B (completion counted on the LEADER's barrier);
+//   warp 10      scale loader: own A-row scale tiles and the scale tiles of all 256 B rows, bulk copies into the ring;
+//                a ring slot is free as soon as the movers have carried it to TMEM, so the loads run two rings ahead;
+//   warps 1, 11  MMA issuers, leader CTA only, taking the K-steps in turn under a baton: four K = 64 pair-MMAs per
+//                step; ONE multicast tcgen05.commit per step frees operand stage and TMEM scale slot in BOTH CTAs;
+//   warps 6..9   scale movers: shared memory -> registers -> own TMEM lane quadrant (tcgen05.st); they arrive on the
+//                leader's full barrier of the stage, the same one the operand bytes complete, so the issuer waits once;
+//   warps 2..5   epilogue of the CTA's own 128 x 256 half tile: accumulator -> registers (packed bf16) -> hand the
+//                accumulator back -> swizzled staging -> TMA stores (or reduce-adds when accumulating).
 // A-row scales are per CTA; every CTA needs the scales of all 256 B rows.
 #include <cuda_bf16.h>
 
@@ -33,7 +36,7 @@ constexpr uint32_t kStageB = 2 * kAB;                       // 32 KB: A rows + B
 constexpr int kSfSlotsP = kStagesP;                         // scale ring: shared-memory slot i feeds TMEM slot i; same ring
                                                             // index as the operand stages so ONE commit frees both
 constexpr uint32_t kSfSlotB = kSfaB + kSfbB;                // 3 KB
-constexpr uint32_t kEpiBuf = 2048;                          // epilogue staging: 32 rows x 64 B, two buffers per epilogue warp
+constexpr uint32_t kEpiBuf = 2048;                          // epilogue staging: 32 rows x 64 B, two buffers per epilogue warp (4 warps)
 constexpr uint32_t kEpiB = 4 * 2 * kEpiBuf;
 constexpr uint32_t kBarB = 256;
 // The dynamic shared-memory window is at least 256-byte aligned, so rounding its base up to 1024 costs at most 768 bytes.
