@@ -117,6 +117,8 @@ gemm_mxf4_pair_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_c
     cluster_sync_all();                                     // both CTAs' barriers exist before anyone signals across
     tc_fence_after_sync();
     const uint32_t tmem_base = *tmem_slot;
+    pdl_launch_dependents();                                // the next kernel of the stream may set itself up behind this one
+    pdl_wait();                                             // everything above overlapped the previous kernel's tail; its data is needed now
 
     if (warp == 0) {
         // ------------------------------------------------------------------ TMA producer (both CTAs)
@@ -412,8 +414,13 @@ cudaError_t launch_gemm_pair(const GemmArgs& a, cudaStream_t stream) {
     const int pairs = tiles < sms / 2 ? tiles : sms / 2;
     p.c_tma = a.has_tmap_c ? 1 : 0;
     p.accumulate = a.accumulate;
-    gemm_mxf4_pair_kernel<<<2 * pairs, kThreadsP, kSmemP, stream>>>(a.tmap_a, a.tmap_b_half, a.tmap_c, p);
-    return cudaGetLastError();
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3(2 * pairs); cfg.blockDim = dim3(kThreadsP); cfg.dynamicSmemBytes = kSmemP; cfg.stream = stream;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr; cfg.numAttrs = 1;
+    return cudaLaunchKernelEx(&cfg, gemm_mxf4_pair_kernel, a.tmap_a, a.tmap_b_half, a.tmap_c, p);
 }
 
 }  // namespace mx

@@ -26,6 +26,13 @@ __device__ __forceinline__ bool elect_one() {
     return pred != 0;
 }
 
+// Programmatic dependent launch: a kernel launched with the programmatic-serialisation attribute may start while
+// its predecessor in the stream is still running.  pdl_launch_dependents lets the successor's CTAs be scheduled as
+// soon as resources free up; pdl_wait blocks until the predecessor grid has completed and its writes are visible
+// (a no-op for a kernel launched without the attribute).
+__device__ __forceinline__ void pdl_launch_dependents() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
+__device__ __forceinline__ void pdl_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
+
 // ---------------------------------------------------------------- mbarrier
 __device__ __forceinline__ void mbar_init(uint64_t* bar, uint32_t count) {
     asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(smem_u32(bar)), "r"(count));

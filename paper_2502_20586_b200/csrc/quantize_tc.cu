@@ -179,6 +179,8 @@ quantize_tc_kernel(const __grid_constant__ QMaps maps, const __grid_constant__ Q
     __syncthreads();
     tc_fence_after_sync();
     const uint32_t tmem_base = *tmem_slot;
+    pdl_launch_dependents();                            // the next kernel of the stream may set itself up behind this one
+    pdl_wait();                                         // the set-up above overlapped the previous kernel's tail; its data is needed now
 
     if (warp == 0) {
         // ------------------------------------------------------------------ TMA producer
@@ -484,17 +486,17 @@ cudaError_t launch_quantize_tc_group(const QuantArgs* a, int n, bool dump_y, cud
         w.d_minor = step % w.minor_count;
     }
     const bool wide = p.g == 256;
-    if (dump_y) {
-        if (wide) quantize_tc_kernel<kModeDump, 2><<<grid, kThreadsQ, kSmemQ, stream>>>(maps, p);
-        else quantize_tc_kernel<kModeDump, 1><<<grid, kThreadsQ, kSmemQ, stream>>>(maps, p);
-    } else if (a[0].rounding == 0) {
-        if (wide) quantize_tc_kernel<kModeSR, 2><<<grid, kThreadsQ, kSmemQ, stream>>>(maps, p);
-        else quantize_tc_kernel<kModeSR, 1><<<grid, kThreadsQ, kSmemQ, stream>>>(maps, p);
-    } else {
-        if (wide) quantize_tc_kernel<kModeRN, 2><<<grid, kThreadsQ, kSmemQ, stream>>>(maps, p);
-        else quantize_tc_kernel<kModeRN, 1><<<grid, kThreadsQ, kSmemQ, stream>>>(maps, p);
-    }
-    return cudaGetLastError();
+    void (*kernel)(QMaps, QParams);
+    if (dump_y) kernel = wide ? quantize_tc_kernel<kModeDump, 2> : quantize_tc_kernel<kModeDump, 1>;
+    else if (a[0].rounding == 0) kernel = wide ? quantize_tc_kernel<kModeSR, 2> : quantize_tc_kernel<kModeSR, 1>;
+    else kernel = wide ? quantize_tc_kernel<kModeRN, 2> : quantize_tc_kernel<kModeRN, 1>;
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3(grid); cfg.blockDim = dim3(kThreadsQ); cfg.dynamicSmemBytes = kSmemQ; cfg.stream = stream;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr; cfg.numAttrs = 1;
+    return cudaLaunchKernelEx(&cfg, kernel, maps, p);
 }
 
 cudaError_t launch_quantize_tc(const QuantArgs& a, bool dump_y, cudaStream_t stream) {
