@@ -21,7 +21,8 @@
 //
 //   warp 0        TMA producer (two 64-column x 128-row boxes per tile, 128-byte swizzle, 4-stage ring)
 //   warp 1        MMA issuer (8 K=16 MMAs per tile into one of four 128-column TMEM accumulators)
-//   warps 2..17   epilogue, four groups of four warps on alternate tiles: warp = TMEM lane quadrant, a thread owns one
+//   warps 2, 3    idle: they complete warp group 0, which hands registers (setmaxnreg) to the epilogue groups
+//   warps 4..19   epilogue, four groups of four warps on alternate tiles: warp = TMEM lane quadrant, a thread owns one
 //                 output row of the tile: tcgen05.ld 32 columns at a time, scale / SR / pack / store per MX block
 // Every mbarrier wait is bounded; on expiry the CTA records a status word and unwinds.
 #include <cuda_bf16.h>
@@ -42,7 +43,7 @@ constexpr uint32_t kSmemQ = kStagesQ * kTileBytes + 2 * kTBytes + 1024 + 256;   
 constexpr int kAccBufs = 4;                         // 4 x 128 TMEM columns
 constexpr int kEpiGroups = 4;                       // epilogue warp groups (one warp per TMEM lane quadrant), on alternate tiles
 constexpr int kEpiWarps = 4 * kEpiGroups;
-constexpr int kThreadsQ = (2 + kEpiWarps) * 32;
+constexpr int kThreadsQ = (4 + kEpiWarps) * 32;    // warp group 0: producer, MMA issuer, two idle warps; then the epilogue warp groups
 
 struct QView {                 // one operand view: output operand [R, K] read from x [rows, cols]
     int64_t R, K;
@@ -182,6 +183,7 @@ quantize_tc_kernel(const __grid_constant__ QMaps maps, const __grid_constant__ Q
     pdl_launch_dependents();                            // the next kernel of the stream may set itself up behind this one
     pdl_wait();                                         // the set-up above overlapped the previous kernel's tail; its data is needed now
 
+    if (warp < 4) reg_dealloc<64>(); else reg_alloc<112>();     // warp group 0 gives registers to the epilogue groups
     if (warp == 0) {
         // ------------------------------------------------------------------ TMA producer
         if (lane == 0) {
@@ -244,13 +246,13 @@ quantize_tc_kernel(const __grid_constant__ QMaps maps, const __grid_constant__ Q
             }
             if (!ok) *abort_flag = 1;
         }
-    } else {
+    } else if (warp >= 4) {
         // ------------------------------------------------------------------ epilogue
         // Four groups of four warps take alternate tiles; inside a group a warp owns one TMEM lane quadrant, i.e. a
         // thread owns one output row of the tile: four MX blocks, 64 bytes of codes, 4 scale bytes.  The SR draws of a
         // block are computed while the block before it is rounded (for a tile's first block: at the end of the tile
         // before); they depend only on element indices.
-        const int e = warp - 2;
+        const int e = warp - 4;
         const int q = warp & 3;                      // TMEM lane quadrant this warp may read
         const int grp = e >> 2;
         const float cg = p.g == 32 ? 0.17677669529663687f : p.g == 128 ? 0.08838834764831845f : 1.0f;
