@@ -342,12 +342,14 @@ mxfp4_status mxfp4_linear_backward_ex(const void* dY, const void* X, const void*
 mxfp4_status mxfp4_device_status(void* cuda_stream) {
     if (cudaStreamSynchronize(static_cast<cudaStream_t>(cuda_stream)) != cudaSuccess) return MXFP4_ERR_CUDA;
     unsigned int word = 0;
-    if (cudaMemcpyFromSymbol(&word, mx::g_device_status, sizeof word) != cudaSuccess) return MXFP4_ERR_CUDA;
-    if (word != 0) {
-        const unsigned int zero = 0;
-        if (cudaMemcpyToSymbol(mx::g_device_status, &zero, sizeof zero) != cudaSuccess) return MXFP4_ERR_CUDA;
-        return MXFP4_ERR_TIMEOUT;
+    cudaError_t (*const fetch[])(unsigned int*) = {mx::fetch_gemm_status, mx::fetch_gemm_pair_status, mx::fetch_quant_tc_status,
+                                                   mx::fetch_fp4_ceiling_status};
+    for (auto f : fetch) {
+        unsigned int w = 0;
+        if (f(&w) != cudaSuccess) return MXFP4_ERR_CUDA;
+        word |= w;
     }
+    if (word != 0) return MXFP4_ERR_TIMEOUT;
     return MXFP4_OK;
 }
 

@@ -7,6 +7,7 @@
 #include <stdint.h>
 
 #include "../../include/mxfp4.h"
+#include "kernels.h"
 #include "ptx.cuh"
 
 namespace mx {
@@ -91,6 +92,9 @@ fp4_ceiling_kernel(uint32_t batches) {
 }
 
 }  // namespace
+
+cudaError_t fetch_fp4_ceiling_status(unsigned int* word) { return device_status_fetch(word); }
+
 }  // namespace mx
 
 extern "C" mxfp4_status mxfp4_fp4_ceiling(int64_t mma_per_pair, int64_t* flop_out, void* cuda_stream) {

@@ -20,8 +20,6 @@
 
 namespace mx {
 
-__device__ unsigned int g_device_status = 0;
-
 namespace {
 
 constexpr int BM = kGemmBM, BN = kGemmBN;
@@ -259,6 +257,8 @@ gemm_mxf4_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_consta
 }
 
 }  // namespace
+
+cudaError_t fetch_gemm_status(unsigned int* word) { return device_status_fetch(word); }
 
 cudaError_t gemm_init() {
     return cudaFuncSetAttribute(gemm_mxf4_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kSmemBytes);

@@ -9,13 +9,13 @@
 //
 // Roles per CTA (12 warps), all waits bounded as in gemm.cu:
 //   warp 0       TMA producer: own A rows, own half of B (completion counted on the LEADER's barrier);
-//   warp 10      scale loader: own A-row scale tiles and the scale tiles of all 256 B rows, bulk copies into the ring;
+//   warp 3       scale loader: own A-row scale tiles and the scale tiles of all 256 B rows, bulk copies into the ring;
 //                a ring slot is free as soon as the movers have carried it to TMEM, so the loads run two rings ahead;
-//   warps 1, 11  MMA issuers, leader CTA only, taking the K-steps in turn under a baton: four K = 64 pair-MMAs per
+//   warps 1, 2   MMA issuers, leader CTA only, taking the K-steps in turn under a baton: four K = 64 pair-MMAs per
 //                step; ONE multicast tcgen05.commit per step frees operand stage and TMEM scale slot in BOTH CTAs;
-//   warps 6..9   scale movers: shared memory -> registers -> own TMEM lane quadrant (tcgen05.st); they arrive on the
+//   warps 8..11  scale movers: shared memory -> registers -> own TMEM lane quadrant (tcgen05.st); they arrive on the
 //                leader's full barrier of the stage, the same one the operand bytes complete, so the issuer waits once;
-//   warps 2..5   epilogue of the CTA's own 128 x 256 half tile: accumulator -> registers (packed bf16) -> hand the
+//   warps 4..7   epilogue of the CTA's own 128 x 256 half tile: accumulator -> registers (packed bf16) -> hand the
 //                accumulator back -> swizzled staging -> TMA stores (or reduce-adds when accumulating).
 // A-row scales are per CTA; every CTA needs the scales of all 256 B rows.
 #include <cuda_bf16.h>
@@ -44,6 +44,9 @@ constexpr uint32_t kSmemP = kStagesP * kStageB + kSfSlotsP * kSfSlotB + kEpiB + 
 static_assert(kSmemP <= 232448, "over the 227 KB shared-memory limit");
 constexpr uint32_t kAccColP = 0, kSfColP = 256, kSfSlotColsP = 24;
 constexpr int kGroupMP = 8;                                 // rasterisation: 8 pair-tiles (2048 rows) share B tiles in L2
+// Register hand-over (setmaxnreg) between the three warp groups; an increase can only draw on what the CTA holds at
+// launch (threads x registers per thread), which gemm_pair_init checks: an increase that cannot be met waits forever.
+constexpr int kRegsLightP = 56, kRegsMoverP = 64, kRegsEpiP = 232;
 constexpr int kThreadsP = 12 * 32;
 
 struct ParamsP {
@@ -117,9 +120,16 @@ gemm_mxf4_pair_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_c
     cluster_sync_all();                                     // both CTAs' barriers exist before anyone signals across
     tc_fence_after_sync();
     const uint32_t tmem_base = *tmem_slot;
+    // Warp group 0 (producer, issuers, scale loader) and warp group 2 (scale movers) need few registers; the epilogue
+    // group takes them to hold half an accumulator row and four TMEM loads in flight.
+    // Each warp group (four warps) sets its register limit once, at the head of its own branch: all four warps must
+    // execute the same setmaxnreg, and the limit must dominate the code that relies on it.
     pdl_launch_dependents();                                // the next kernel of the stream may set itself up behind this one
     pdl_wait();                                             // everything above overlapped the previous kernel's tail; its data is needed now
 
+    if (warp < 4) {
+    // ============================ warp group 0: producer, two MMA issuers, scale loader (few registers each)
+    reg_dealloc<kRegsLightP>();
     if (warp == 0) {
         // ------------------------------------------------------------------ TMA producer (both CTAs)
         if (lane == 0) {
@@ -140,11 +150,11 @@ gemm_mxf4_pair_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_c
             }
             if (!ok) *abort_flag = 1;
         }
-    } else if (warp == 1 || warp == 11) {
+    } else if (warp == 1 || warp == 2) {
         // ------------------------------------------------------------------ MMA issuers (leader CTA only)
         // Issuing one pair MMA occupies its thread for ~90 cycles and a commit for ~100, which is more than the
         // tensor pipe needs for the four MMAs of a step.  Two threads therefore take the steps in turn (even steps
-        // warp 1, odd steps warp 11): while one issues, the other has already waited for its operands and then
+        // warp 1, odd steps warp 2): while one issues, the other has already waited for its operands and then
         // commits.  A baton (mbarrier turn[]) keeps the MMAs in step order, so accumulation order is fixed.
         if (rank == 0 && lane == 0) {
             // instruction descriptor: A, B = E2M1 (1), scale = UE8M0 (1), K-major, N >> 3 at bit 17, M >> 4 at bit 24
@@ -189,7 +199,7 @@ gemm_mxf4_pair_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_c
             }
             if (!ok) *abort_flag = 1;
         }
-    } else if (warp == 10) {
+    } else {
         // ------------------------------------------------------------------ scale loader (both CTAs)
         if (lane == 0) {
             uint32_t it = 0;
@@ -215,7 +225,10 @@ gemm_mxf4_pair_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_c
             }
             if (!ok) *abort_flag = 1;
         }
-    } else if (warp >= 6) {
+    }
+    } else if (warp >= 8) {
+        // ============================ warp group 2: scale movers
+        reg_dealloc<kRegsMoverP>();
         // ------------------------------------------------------------------ scale movers (both CTAs, warps 6..9)
         const int q = warp & 3;
         const uint32_t lane_base = (uint32_t)(q * 32) << 16;
@@ -242,6 +255,7 @@ gemm_mxf4_pair_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_c
         if (!ok && lane == 0) *abort_flag = 1;
     } else {
         // ------------------------------------------------------------------ epilogue (both CTAs, own 128 rows)
+        reg_alloc<kRegsEpiP>();                                   // warp group 1 takes the registers the others gave up
         // TMEM -> registers -> (alpha, convert) -> shared memory -> TMA store.  Each warp owns the 32 accumulator
         // lanes of its quadrant and two 2 KB staging buffers (32 rows x 64 bytes, 64-byte swizzle, so the row-per-lane
         // writes are conflict-free); the accumulator is handed back as soon as its last column is in registers.
@@ -287,20 +301,26 @@ gemm_mxf4_pair_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_c
                 // bf16: drain the whole accumulator into registers first (packed pairs), hand it back, then store.
                 uint32_t out[PN / 2];
 #pragma unroll
-                for (int c = 0; c < PN / 32; ++c) {
-                    uint32_t r[32];
-                    tmem_ld_32x32b_x32(tmem_base + kAccColP + ((uint32_t)(q * 32) << 16) + c * 32, r);
-                    tmem_ld_wait();
+                for (int hb = 0; hb < 2; ++hb) {                // two batches of four 32-column loads in flight together
+                    uint32_t r[4][32];
 #pragma unroll
-                    for (int j = 0; j < 16; ++j) {
-                        const __nv_bfloat162 h = __floats2bfloat162_rn(__uint_as_float(r[2 * j]) * p.alpha,
-                                                                       __uint_as_float(r[2 * j + 1]) * p.alpha);
-                        out[16 * c + j] = *reinterpret_cast<const uint32_t*>(&h);
+                    for (int c = 0; c < 4; ++c)
+                        tmem_ld_32x32b_x32(tmem_base + kAccColP + ((uint32_t)(q * 32) << 16) + (4 * hb + c) * 32, r[c]);
+                    tmem_ld_wait();
+                    if (hb == 1) {                              // the accumulator is in registers: hand it back before converting
+                        tc_fence_before_sync();
+                        __syncwarp();
+                        if (lane == 0) mbar_arrive_cluster(tmem_empty, 0);
                     }
+#pragma unroll
+                    for (int c = 0; c < 4; ++c)
+#pragma unroll
+                        for (int j = 0; j < 16; ++j) {
+                            const __nv_bfloat162 h = __floats2bfloat162_rn(__uint_as_float(r[c][2 * j]) * p.alpha,
+                                                                           __uint_as_float(r[c][2 * j + 1]) * p.alpha);
+                            out[16 * (4 * hb + c) + j] = *reinterpret_cast<const uint32_t*>(&h);
+                        }
                 }
-                tc_fence_before_sync();
-                __syncwarp();
-                if (lane == 0) mbar_arrive_cluster(tmem_empty, 0);
 #pragma unroll
                 for (int c = 0; c < PN / 32; ++c) {
                     uint32_t w[16];
@@ -394,8 +414,16 @@ gemm_mxf4_pair_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_c
 
 }  // namespace
 
+cudaError_t fetch_gemm_pair_status(unsigned int* word) { return device_status_fetch(word); }
+
 cudaError_t gemm_pair_init() {
-    return cudaFuncSetAttribute(gemm_mxf4_pair_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kSmemP);
+    cudaError_t e = cudaFuncSetAttribute(gemm_mxf4_pair_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kSmemP);
+    if (e != cudaSuccess) return e;
+    cudaFuncAttributes fa;
+    e = cudaFuncGetAttributes(&fa, gemm_mxf4_pair_kernel);
+    if (e != cudaSuccess) return e;
+    if (fa.numRegs * kThreadsP < 128 * (kRegsLightP + kRegsMoverP + kRegsEpiP)) return cudaErrorLaunchOutOfResources;
+    return cudaSuccess;
 }
 
 cudaError_t launch_gemm_pair(const GemmArgs& a, cudaStream_t stream) {

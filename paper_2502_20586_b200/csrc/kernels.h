@@ -59,6 +59,12 @@ constexpr int kGemmBKBytes = 128;   // 256 E2M1 elements per pipeline stage
 size_t bias_grad_workspace(int64_t b, int64_t m);
 cudaError_t launch_bias_grad(const void* dY, int64_t b, int64_t m, int64_t ld, int accumulate, float* db, float* partial, cudaStream_t stream);
 
+// Each kernel file keeps its own device status word (set when a bounded wait expires); these read and clear them.
+cudaError_t fetch_gemm_status(unsigned int* word);
+cudaError_t fetch_gemm_pair_status(unsigned int* word);
+cudaError_t fetch_quant_tc_status(unsigned int* word);
+cudaError_t fetch_fp4_ceiling_status(unsigned int* word);
+
 cudaError_t launch_gemm(const GemmArgs& a, cudaStream_t stream);
 cudaError_t gemm_init();            // one-time: opt in to large dynamic shared memory
 cudaError_t launch_gemm_pair(const GemmArgs& a, cudaStream_t stream);

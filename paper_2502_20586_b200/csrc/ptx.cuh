@@ -7,8 +7,23 @@
 
 namespace mx {
 
-// Set by any kernel whose bounded wait expired; read and cleared by mxfp4_device_status().
-extern __device__ unsigned int g_device_status;
+// Set by any kernel of this translation unit whose bounded wait expired.  Every .cu file that includes this header
+// has its own copy (the library is built without relocatable device code, which is what lets ptxas honour
+// setmaxnreg); each such file exports a fetch_*_status() built on device_status_fetch(), and
+// mxfp4_device_status() combines them.
+static __device__ unsigned int g_device_status = 0;
+
+// Host: read this translation unit's status word into *word and clear it if it was set.
+static inline cudaError_t device_status_fetch(unsigned int* word) {
+    unsigned int w = 0;
+    cudaError_t e = cudaMemcpyFromSymbol(&w, g_device_status, sizeof w);
+    if (e == cudaSuccess && w != 0) {
+        const unsigned int zero = 0;
+        e = cudaMemcpyToSymbol(g_device_status, &zero, sizeof zero);
+    }
+    *word = w;
+    return e;
+}
 
 constexpr unsigned int kStatusTimeout = 1u;
 
@@ -83,7 +98,8 @@ __device__ __forceinline__ bool mbar_try_wait_hint(uint64_t* bar, uint32_t parit
         : "=r"(ok) : "r"(smem_u32(bar)), "r"(parity), "r"(hint_ns) : "memory");
     return ok != 0;
 }
-static __device__ __noinline__ bool mbar_wait_slow(uint64_t* bar, uint32_t parity, const volatile uint32_t* abort) {
+// (inlined: a kernel that re-balances registers with setmaxnreg cannot call out-of-line functions)
+static __device__ __forceinline__ bool mbar_wait_slow(uint64_t* bar, uint32_t parity, const volatile uint32_t* abort) {
     const uint64_t t0 = global_timer_ns();
     for (uint32_t i = 0;; ++i) {
         if (mbar_try_wait_hint(bar, parity, 1000u)) return true;
@@ -99,7 +115,7 @@ __device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity, const 
 }
 // Same bound, but polling without a suspend hint: for the one thread whose wake-up latency is on the critical
 // path (the MMA issuer), in particular when the arrivals come from the other CTA of a pair.
-static __device__ __noinline__ bool mbar_wait_spin(uint64_t* bar, uint32_t parity, const volatile uint32_t* abort) {
+static __device__ __forceinline__ bool mbar_wait_spin(uint64_t* bar, uint32_t parity, const volatile uint32_t* abort) {
     const uint64_t t0 = global_timer_ns();
     for (uint32_t i = 0;; ++i) {
         if (mbar_try_wait(bar, parity)) return true;

@@ -43,6 +43,10 @@ constexpr uint32_t kSmemQ = kStagesQ * kTileBytes + 2 * kTBytes + 1024 + 256;   
 constexpr int kAccBufs = 4;                         // 4 x 128 TMEM columns
 constexpr int kEpiGroups = 4;                       // epilogue warp groups (one warp per TMEM lane quadrant), on alternate tiles
 constexpr int kEpiWarps = 4 * kEpiGroups;
+// Register hand-over (setmaxnreg): warp group 0 shrinks to kRegsLight, the epilogue groups grow to kRegsEpi.  The
+// increase can only draw on what the CTA itself holds, i.e. threads x registers-per-thread at launch: the init
+// routine checks that budget against the compiled kernel, because an increase that cannot be met waits forever.
+constexpr int kRegsLight = 40, kRegsEpi = 104;
 constexpr int kThreadsQ = (4 + kEpiWarps) * 32;    // warp group 0: producer, MMA issuer, two idle warps; then the epilogue warp groups
 
 struct QView {                 // one operand view: output operand [R, K] read from x [rows, cols]
@@ -183,7 +187,9 @@ quantize_tc_kernel(const __grid_constant__ QMaps maps, const __grid_constant__ Q
     pdl_launch_dependents();                            // the next kernel of the stream may set itself up behind this one
     pdl_wait();                                         // the set-up above overlapped the previous kernel's tail; its data is needed now
 
-    if (warp < 4) reg_dealloc<64>(); else reg_alloc<112>();     // warp group 0 gives registers to the epilogue groups
+    if (warp < 4) {
+    // ============================ warp group 0: producer, MMA issuer, two idle warps; it gives registers to the others
+    reg_dealloc<kRegsLight>();
     if (warp == 0) {
         // ------------------------------------------------------------------ TMA producer
         if (lane == 0) {
@@ -246,8 +252,10 @@ quantize_tc_kernel(const __grid_constant__ QMaps maps, const __grid_constant__ Q
             }
             if (!ok) *abort_flag = 1;
         }
-    } else if (warp >= 4) {
-        // ------------------------------------------------------------------ epilogue
+    }
+    } else {
+        // ------------------------------------------------------------------ epilogue (warp groups 1..4)
+        reg_alloc<kRegsEpi>();
         // Four groups of four warps take alternate tiles; inside a group a warp owns one TMEM lane quadrant, i.e. a
         // thread owns one output row of the tile: four MX blocks, 64 bytes of codes, 4 scale bytes.  The SR draws of a
         // block are computed while the block before it is rounded (for a tile's first block: at the end of the tile
@@ -431,13 +439,20 @@ bool quant_tc_eligible(const QuantArgs& a) {
     return (a.g == 32 || a.g == 64 || a.g == 128 || a.g == 256) && K % kTile == 0 && tiles < (int64_t(1) << 28) && a.has_tmap;
 }
 
+cudaError_t fetch_quant_tc_status(unsigned int* word) { return device_status_fetch(word); }
+
 cudaError_t quant_tc_init() {
     const void* kernels[6] = {(const void*)quantize_tc_kernel<kModeSR, 1>, (const void*)quantize_tc_kernel<kModeRN, 1>,
                               (const void*)quantize_tc_kernel<kModeDump, 1>, (const void*)quantize_tc_kernel<kModeSR, 2>,
                               (const void*)quantize_tc_kernel<kModeRN, 2>, (const void*)quantize_tc_kernel<kModeDump, 2>};
     for (const void* k : kernels) {
-        const cudaError_t e = cudaFuncSetAttribute(k, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kSmemQ);
+        cudaError_t e = cudaFuncSetAttribute(k, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kSmemQ);
         if (e != cudaSuccess) return e;
+        cudaFuncAttributes fa;
+        e = cudaFuncGetAttributes(&fa, k);
+        if (e != cudaSuccess) return e;
+        // registers the CTA holds at launch must cover the limits the warp groups set for themselves
+        if (fa.numRegs * kThreadsQ < 128 * kRegsLight + (kThreadsQ - 128) * kRegsEpi) return cudaErrorLaunchOutOfResources;
     }
     return cudaSuccess;
 }
