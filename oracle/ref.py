@@ -36,6 +36,10 @@ _lib.orc_e8m0_from_amax.argtypes = [C.c_float]
 _lib.orc_e8m0_from_amax.restype = C.c_uint32
 _lib.orc_sr_round.argtypes = [C.c_double, C.c_uint32]
 _lib.orc_sr_round.restype = C.c_uint32
+_lib.orc_sr16_draw.argtypes = [_u64, C.c_uint32, _u64]
+_lib.orc_sr16_draw.restype = C.c_uint32
+_lib.orc_sr16_round.argtypes = [C.c_double, C.c_uint32]
+_lib.orc_sr16_round.restype = C.c_uint32
 _lib.orc_rn_round.argtypes = [C.c_double]
 _lib.orc_rn_round.restype = C.c_uint32
 _lib.orc_quantize.argtypes = [_f32p, _i64, _i64, C.c_int, _u64, C.c_uint32, _u8p, _u8p]
@@ -63,6 +67,7 @@ _lib.orc_num_threads.restype = C.c_int
 
 ROUND_SR = 0
 ROUND_RN = 1
+ROUND_SR16 = 2      # Algorithm 2 with the 16-bit dither of the second SR reading
 
 
 def num_threads() -> int:
@@ -102,6 +107,14 @@ def e8m0_from_amax(amax: float) -> int:
 
 def sr_round(w: float, r: int) -> int:
     return int(_lib.orc_sr_round(w, r))
+
+
+def sr16_draw(seed: int, stream_tag: int, i: int) -> int:
+    return int(_lib.orc_sr16_draw(seed, stream_tag, i))
+
+
+def sr16_round(w: float, R: int) -> int:
+    return int(_lib.orc_sr16_round(w, R))
 
 
 def rn_round(w: float) -> int:

@@ -293,6 +293,128 @@ def test_sr_monte_carlo_through_philox(ref):
     assert np.all(np.abs(acc / T - 0.75 * y) <= 5 * sigma + X / 512)
 
 
+# --------------------------------------------------------------------------- second SR reading (16-bit dither)
+
+def _rev(v, bits):
+    return int(format(v, "0%db" % bits)[::-1], 2)
+
+
+def test_sr16_draw_layout(ref):
+    """The 16-bit dithers of four consecutive elements come from one Philox word: bytes (b2, b0) and (b3, b1),
+    odd elements bit-reversed, so the leading eight bits of the four dithers are four different bytes."""
+    seed = 0x0123456789ABCDEF
+    key = [seed & 0xFFFFFFFF, seed >> 32]
+    for tag, h in ((1, 0), (2, 3), (3, 4), (4, (2**33 + 8) // 4)):
+        i = 4 * h
+        out = ref.philox4x32_10([(i >> 4) & 0xFFFFFFFF, (i >> 4) >> 32, tag, 1], key)
+        word = int(out[(i >> 2) & 3])
+        b = [(word >> (8 * k)) & 0xFF for k in range(4)]
+        d = [ref.sr16_draw(seed, tag, i + j) for j in range(4)]
+        assert d[0] == 256 * b[2] + b[0] and d[2] == 256 * b[3] + b[1]
+        assert d[1] == _rev(d[0], 16) and d[3] == _rev(d[2], 16)
+        assert [x >> 8 for x in d] == [b[2], _rev(b[0], 8), b[3], _rev(b[1], 8)]
+        # the same bytes the 8-bit reading draws for these four elements
+        assert [ref.sr_draw(seed, tag, i + j) for j in range(4)] == b
+    n = 1 << 15
+    d = np.array([ref.sr16_draw(7, 1, i) for i in range(n)])
+    for top in (d >> 8, d & 0xFF, (d >> 4) & 0xFF):
+        counts = np.bincount(top, minlength=256)
+        chi2 = ((counts - n / 256.0) ** 2 / (n / 256.0)).sum()
+        assert chi2 < 255 + 6 * np.sqrt(2 * 255)
+    # leading bytes of paired elements are uncorrelated
+    a, b2 = (d[0::4] >> 8).astype(float), (d[1::4] >> 8).astype(float)
+    assert abs(np.corrcoef(a, b2)[0, 1]) < 5 / np.sqrt(len(a))
+
+
+def test_sr16_law_by_enumeration(ref):
+    """P(up) = floor(65536 frac) / 65536: the smallest dither that rounds up is 65536 - floor(65536 frac);
+    E[SR16(w)] lies in (w - gap / 65536, w]; the hand-worked cases of the 8-bit reading hold to 2^-16."""
+    def first_up(w):                                           # monotone in R: bisection over [0, 65536]
+        lo = max(i for i, v in enumerate(GRID) if v <= abs(w))
+        a, b = 0, 65536                                        # invariant: R < a rounds down, R >= b rounds up
+        while a < b:
+            mid = (a + b) // 2
+            if (ref.sr16_round(w, mid) & 7) == lo + 1: b = mid
+            else: a = mid + 1
+        return a
+    rng = np.random.default_rng(21)
+    ws = list(rng.uniform(0, 5.9999, 300)) + [5.25, 0.75, 0.225, 1.65, 5.4, 3.0 + 2.0 ** -16, 4 + 2.0 ** -14, 0.5 - 2.0 ** -18, 1e-12]
+    for w in ws:
+        lo = max(v for v in GRID if v <= w)
+        hi = min(v for v in GRID if v > w)
+        F = int(np.floor((w - lo) / (hi - lo) * 65536))
+        for sgn in (1.0, -1.0):
+            t = first_up(sgn * w)
+            assert t == 65536 - F or (F == 0 and t == 65536)
+            if 0 < t < 65536:                                   # both sides of the threshold, and monotone beyond
+                assert ref.e2m1_value(ref.sr16_round(sgn * w, t - 1)) == sgn * lo
+                assert ref.e2m1_value(ref.sr16_round(sgn * w, t)) == sgn * hi
+                assert ref.e2m1_value(ref.sr16_round(sgn * w, 65535)) == sgn * hi
+            assert ref.e2m1_value(ref.sr16_round(sgn * w, 0)) == sgn * lo
+        mean = lo + (hi - lo) * F / 65536.0
+        assert w - (hi - lo) / 65536.0 < mean <= w
+    # full enumeration for the worked SR cases: two outcomes, probability and mean as printed, variance (c - a)(a - f)
+    for tok in _lines("worked_blocks.txt"):
+        if tok[0] != "sr":
+            continue
+        w, lo, hi, p_up = (float(t) for t in tok[1:5])
+        vals = np.array([ref.e2m1_value(ref.sr16_round(w, R)) for R in range(65536)])
+        assert set(vals) <= {lo, hi}
+        assert abs((vals == hi).mean() - p_up) <= 2.0 ** -16 + 1e-12
+        assert abs(vals.mean() - w) <= abs(hi - lo) * 2.0 ** -16 + 1e-12
+        assert abs(vals.var() - abs(hi - w) * abs(w - lo)) <= (hi - lo) ** 2 * 2.0 ** -15
+    # grid points are fixed points, the sign of zero is kept, |w| >= 6 saturates
+    for c in range(16):
+        v = ref.e2m1_value(c)
+        assert all(ref.sr16_round(v, R) == c for R in (0, 1, 32768, 65535)) or c == 8
+    assert ref.sr16_round(-0.0, 65535) == 8 and ref.sr16_round(0.0, 65535) == 0
+    assert ref.sr16_round(6.5, 0) == 7 and ref.sr16_round(-7.0, 0) == 15
+
+
+def test_quantize_blocks_sr16(ref):
+    """Algorithm 2 with the 16-bit reading: same scales as the 8-bit reading, codes from (w, dither by index);
+    unbiased through the real generator, and paired elements round independently."""
+    seed, tag = 99, 3
+    rng = np.random.default_rng(4)
+    y = (rng.standard_normal((4, 96)) * np.array([[1e-3], [1.0], [37.0], [1e4]])).astype(np.float32)
+    y[1, 32:64] = 0.0
+    codes, scales = ref.quantize(y, ref.ROUND_SR16, seed, tag)
+    assert np.array_equal(scales, ref.quantize(y, ref.ROUND_SR, seed, tag)[1])
+    for r in range(4):
+        for b in range(3):
+            V = y[r, 32 * b:32 * b + 32].astype(np.float64)
+            w = 0.75 * V / 2.0 ** (int(scales[r, b]) - 127)
+            for i in range(32):
+                idx = r * 96 + 32 * b + i
+                assert codes[r, 32 * b + i] == ref.sr16_round(w[i], ref.sr16_draw(seed, tag, idx))
+    # row_ids shift the element index that keys the dither
+    sub = ref.quantize(y[2:3], ref.ROUND_SR16, seed, tag, row_ids=np.array([2]))[0]
+    assert np.array_equal(sub[0], codes[2])
+    y = rng.standard_normal((8, 64)).astype(np.float32)
+    T = 3000
+    acc = np.zeros(y.shape)
+    err = np.zeros((T,) + y.shape)
+    for t in range(T):
+        c, sc = ref.quantize(y, ref.ROUND_SR16, 1234, t)
+        dq = ref.dequantize(c, sc)
+        acc += dq
+        err[t] = dq - 0.75 * y
+    X = 2.0 ** (sc.astype(np.float64) - 127).repeat(32, axis=1)
+    assert np.all(np.abs(acc / T - 0.75 * y) <= 5 * X / np.sqrt(T) + X * 2.0 ** -15)
+    e = err / X
+    for j in (0, 2):                                           # elements (4h, 4h+1) and (4h+2, 4h+3) share 16 bits
+        a, b2 = e[:, :, j::4], e[:, :, j + 1::4]
+        corr = ((a - a.mean(0)) * (b2 - b2.mean(0))).mean(0) / (a.std(0) * b2.std(0) + 1e-30)
+        assert np.abs(corr).max() < 6 / np.sqrt(T)
+    # Algorithm 3 carries the 16/9 in this reading too
+    dY = wl.grad_like(rng, (32, 32), 1e-3)
+    Xa = wl.activation_like(rng, (32, 32))
+    W = wl.weight_like(rng, (32, 32))
+    ex = wl.bf16_bits_to_f64(dY) @ wl.bf16_bits_to_f64(W)
+    sx = sum(ref.linear_backward(dY, Xa, W, 32, ref.ROUND_SR16, 500 + t)[0] for t in range(48)) / 48
+    assert abs(np.vdot(sx, ex) / np.vdot(ex, ex) - 1.0) < 0.05
+
+
 # --------------------------------------------------------------------------- GEMM and Algorithm 3
 
 def test_gemm_special_cases(ref):
