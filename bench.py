@@ -38,6 +38,7 @@ QUANT_BYTES_PER_ELEM = 2.0 + 0.5 + 1.0 / 32.0   # bf16 in, E2M1 code + E8M0 scal
 # DRAM bytes moved / algorithmic bytes of the GEMM, from one ncu capture (profiles/gemm_mxf4_pair_16384x4096x16384.md:
 # 477.8 MB measured against 312.6 MB of codes, scales and bf16 output); applied to the average launch of the step.
 GEMM_TRAFFIC_OVER_ALGORITHMIC = 1.49
+ROUNDINGS = {"sr": 0, "rn": 1, "sr16": 2}      # the C ABI's and the oracle's rounding selectors
 
 
 def load_peaks():
@@ -106,7 +107,7 @@ class ClockSampler:
 
 
 # ------------------------------------------------------------------------------------------ reference arm
-def oracle_sample(config: str, seed: int = 0, tokens: int = 4096, dw_sample: int = 4096):
+def oracle_sample(config: str, seed: int = 0, tokens: int = 4096, dw_sample: int = 4096, rounding: str = "sr"):
     """A bounded sample of the workload for the CPU oracle: Algorithm 3 on a `tokens`-token slab of the
     attention-output layer, dX in full and dW on up to `dw_sample` sampled rows.  Returns (fn, flops, description, threads)."""
     import numpy as np
@@ -124,9 +125,9 @@ def oracle_sample(config: str, seed: int = 0, tokens: int = 4096, dw_sample: int
     flops = 2 * b_s * layer.n * layer.m + 2 * len(dw_rows) * layer.n * b_s
 
     def run():
-        ref.linear_backward(dY, X, W, g, ref.ROUND_SR, seed, dw_rows=dw_rows)
+        ref.linear_backward(dY, X, W, g, ROUNDINGS[rounding], seed, dw_rows=dw_rows)
 
-    desc = (f"Algorithm 3 (g={g}, SR) on a {b_s}-token slab of the {config} {layer.name} layer (n={layer.n}, m={layer.m}): "
+    desc = (f"Algorithm 3 (g={g}, {rounding.upper()}) on a {b_s}-token slab of the {config} {layer.name} layer (n={layer.n}, m={layer.m}): "
             f"all four operand quantisations, dX in full, dW on {len(dw_rows)} sampled rows; FLOPs = GEMM MACs x 2 actually computed")
     return run, flops, desc, ref.num_threads()
 
@@ -136,7 +137,7 @@ def run_reference(args):
     if rank != 0:
         return
     # each step is a quarter of the cpu_baseline sample (about 2 s), so that 40 steps still end within two minutes
-    run, flops, desc, cores = oracle_sample(args.config, tokens=2048, dw_sample=2048)
+    run, flops, desc, cores = oracle_sample(args.config, tokens=2048, dw_sample=2048, rounding=args.rounding)
     for _ in range(min(args.warmup, 1)):
         run()
     t0 = time.perf_counter()
@@ -211,9 +212,11 @@ def run_gpu(args):
     flops_step = sum(l.flops for l in layers)
     stream = torch.cuda.current_stream()
 
-    def step():
+    rnd = ROUNDINGS[args.rounding]
+
+    def step(rnd=rnd):
         for (layer, dY, X, W, dX, dW) in data:
-            mx.mxfp4_linear_backward(dY, X, W, g, seed, mx.ROUND_SR, out_dtype, dX=dX, dW=dW, workspace=ws)
+            mx.mxfp4_linear_backward(dY, X, W, g, seed, rnd, out_dtype, dX=dX, dW=dW, workspace=ws)
 
     # ---- value: K steps, device-resident inputs
     sampler = ClockSampler(local_rank)
@@ -233,6 +236,7 @@ def run_gpu(args):
 
     legs = set(args.legs.split(","))
     kernels, calls_ms, gemm_tflops, clocks = {}, None, None, None
+    variants = {}
     fp4_peak = BF16_TO_FP4 * peaks["bf16_sustained"]
     if "roofline" in legs:
         # ---- roofline: the same step as its six C-ABI calls per layer, CUDA events around each
@@ -258,14 +262,14 @@ def run_gpu(args):
             for (layer, dY, X, W, dX, dW), ops in zip(data, bufs):
                 for (t, rd, tag, codes, scales) in ops:
                     fn = lambda t=t, rd=rd, tag=tag, codes=codes, scales=scales: mx.mxfp4_rht_sr_quantize(
-                        t, rd, g, seed, tag, mx.ROUND_SR, mx.SF_NATIVE, codes=codes, scales=scales)
+                        t, rd, g, seed, tag, rnd, mx.SF_NATIVE, codes=codes, scales=scales)
                     if record:
                         timed("quant_row" if rd == 1 else "quant_tr", layer.name, t.numel() * QUANT_BYTES_PER_ELEM, fn)
                     else:
                         fn()
                 for (a, bb, out, fl) in ((0, 1, dX, 2 * layer.b * layer.n * layer.m), (2, 3, dW, 2 * layer.m * layer.n * layer.b)):
                     fn = lambda a=a, bb=bb, out=out, ops=ops: mx.mxfp4_gemm(ops[a][3], ops[a][4], ops[bb][3], ops[bb][4],
-                                                                             16.0 / 9.0, out_dtype, C_out=out)
+                                                                             16.0 / 9.0 if rnd != 1 else 1.0, out_dtype, C_out=out)
                     if record:
                         timed("gemm", layer.name, fl, fn)
                     else:
@@ -295,6 +299,22 @@ def run_gpu(args):
                            "frac_of_4x_bf16_burst": gemm_tflops / (BF16_TO_FP4 * peaks["bf16_burst"]),
                            "frac_of_nominal_9pf": gemm_tflops / NOMINAL_FP4_TFLOPS}
         calls_ms = sum(v[0] for v in agg.values()) / k_roof * 1e3
+        # the other stochastic-rounding reading, same step, a short run
+        if args.rounding in ("sr", "sr16"):
+            other = "sr16" if args.rounding == "sr" else "sr"
+            for _ in range(3):
+                step(ROUNDINGS[other])
+            a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            k_var = max(1, min(args.steps, 20))
+            barrier()
+            a.record(stream)
+            for _ in range(k_var):
+                step(ROUNDINGS[other])
+            b.record(stream)
+            barrier()
+            ms_var = a.elapsed_time(b) / k_var
+            variants[other] = {"ms_per_step": ms_var, "value": flops_step / (ms_var * 1e-3) / 1e12, "steps": k_var,
+                               "note": "this rank's step with the other SR reading (8-bit centred dither / 16-bit dither of the hardware convert)"}
 
     clocks = sampler.stop()
     if gemm_tflops is not None:
@@ -340,7 +360,7 @@ def run_gpu(args):
                 stream.wait_event(ev_in[i])
                 if used[0]:
                     stream.wait_event(ev_out[i])                # the previous step's outputs have left the device
-                mx.mxfp4_linear_backward(dY, X, W, g, seed, mx.ROUND_SR, out_dtype, dX=dX, dW=dW, workspace=ws)
+                mx.mxfp4_linear_backward(dY, X, W, g, seed, rnd, out_dtype, dX=dX, dW=dW, workspace=ws)
                 ev_comp[i].record(stream)
                 s_out.wait_event(ev_comp[i])
                 with torch.cuda.stream(s_out):
@@ -375,7 +395,7 @@ def run_gpu(args):
 
     cpu_baseline = None
     if rank == 0 and world == 1 and not args.no_cpu_baseline and "e2e" in legs:
-        run, fl, desc, cores = oracle_sample(args.config)
+        run, fl, desc, cores = oracle_sample(args.config, rounding=args.rounding)
         t0 = time.perf_counter()
         run()
         dt = time.perf_counter() - t0
@@ -386,7 +406,7 @@ def run_gpu(args):
             "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps, "warmup": args.warmup,
             "ms_per_step": ms, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
             "dtype": "mxfp4", "data": "synthetic",
-            "config": {"workload": args.config, "layers": {l.name: [l.b, l.n, l.m] for l in layers}, "g": g, "rounding": "SR",
+            "config": {"workload": args.config, "layers": {l.name: [l.b, l.n, l.m] for l in layers}, "g": g, "rounding": args.rounding.upper(),
                        "out_dtype": "bf16", "flops_per_step": flops_step, "l2": "inputs_exceed_l2",
                        "frac_of_4x_bf16_sustained": value / world / fp4_peak, "frac_of_nominal_9pf": value / world / NOMINAL_FP4_TFLOPS,
                        "step_as_separate_calls_ms": calls_ms},
@@ -400,6 +420,7 @@ def run_gpu(args):
                          "traffic_note": "bytes per average launch = algorithmic bytes x 1.49 (ratio from an ncu capture of the 16384x4096x16384 launch)",
                          "peak_source": f"4 x {peaks['source']} sustained bf16 ({peaks['bf16_sustained']} TFLOP/s); no FP4 peak was measured"},
             "kernels": kernels,
+            "variants": variants,
             "hbm_peak_gbs": peaks["hbm_gbs"], "peaks_source": peaks["source"],
             "cpu_baseline": cpu_baseline,
         }))
@@ -415,6 +436,7 @@ def main():
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--config", default="gpt_6p7b")
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--rounding", default="sr", choices=sorted(ROUNDINGS), help="sr: 8-bit centred dither; sr16: 16-bit dither of the hardware convert; rn: Algorithm 1")
     ap.add_argument("--legs", default="value,roofline,e2e", help="comma list of GPU legs to run (profiling runs use 'value')")
     args = ap.parse_args()
     if args.impl == "reference":

@@ -52,8 +52,9 @@ typedef enum {
     MXFP4_ERR_TIMEOUT = 9     /* a bounded device-side wait expired (see mxfp4_device_status) */
 } mxfp4_status;
 
-/* rounding: Algorithm 2 (3/4 pre-scale + stochastic rounding) or Algorithm 1 (OCP nearest rounding) */
-enum { MXFP4_ROUND_SR = 0, MXFP4_ROUND_RN = 1 };
+/* rounding: Algorithm 2 (3/4 pre-scale + stochastic rounding; SR with an 8-bit dither and a centred threshold,
+ * SR16 with the 16-bit dither of the sm_100a stochastic-rounding convert) or Algorithm 1 (OCP nearest rounding) */
+enum { MXFP4_ROUND_SR = 0, MXFP4_ROUND_RN = 1, MXFP4_ROUND_SR16 = 2 };
 /* scale layout: LINEAR = [rows, K/32] row-major bytes.
  * NATIVE = the tcgen05 scale-factor tiling consumed by mxfp4_gemm: rows padded to 128, K/32 padded to 4;
  * byte of (row r, block k) at ((r/128)*ceil(K/128) + k/4)*512 + (r%32)*16 + ((r%128)/32)*4 + k%4. */
@@ -73,7 +74,11 @@ enum { MXFP4_OUT_BF16 = 0, MXFP4_OUT_FP32 = 1 };
  *              v diag(S) H_g / sqrt(g), H_g the Sylvester Hadamard matrix (Eq. 4), S derived from `seed`.
  *   rounding   MXFP4_ROUND_SR: per 32 values, shared_exp = floor(log2 amax) - 2, then each value is
  *              multiplied by 3/4, divided by 2^shared_exp and stochastically rounded to E2M1 with an 8-bit
- *              Philox4x32-10 draw keyed on (seed, stream_tag, element index).  MXFP4_ROUND_RN: nearest
+ *              Philox4x32-10 draw r keyed on (seed, stream_tag, element index): up iff 256 frac >= r + 1/2.
+ *              MXFP4_ROUND_SR16: the same with a 16-bit dither R, up iff 65536 frac >= 65536 - R (Eq. 2 to
+ *              2^-16); the elements 4h..4h+3 of a row share the Philox word whose bytes the SR mode draws for
+ *              them, b0..b3: R = 256 b2 + b0, its bit reversal, 256 b3 + b1, its bit reversal.  One convert
+ *              instruction rounds four values, which makes this mode the faster one.  MXFP4_ROUND_RN: nearest
  *              rounding (ties to even, saturating at 6) of value / 2^shared_exp, no pre-scale.
  *   seed       drives the sign vector (shared by every operand quantised with the same seed) and SR.
  *   stream_tag separates the SR noise of different operands that share a seed (they must differ between
@@ -113,7 +118,7 @@ MXFP4_API size_t mxfp4_linear_backward_workspace(int64_t b, int64_t m, int64_t n
  *   dY bf16 [b, m], X bf16 [b, n], W bf16 [m, n]  ->  dX [b, n], dW [m, n] (bf16 or fp32, dense).
  *   g divides m and b (the two reduction lengths); with g = 0, m % 128 == 0 and b % 128 == 0.
  *   The four operand views are quantised with stream tags 1..4 (dY, W^T, dY^T, X^T) and one shared sign
- *   vector; dX = alpha Q1 Q2^T, dW = alpha Q3 Q4^T with alpha = 16/9 iff rounding = SR.
+ *   vector; dX = alpha Q1 Q2^T, dW = alpha Q3 Q4^T with alpha = 16/9 iff rounding = SR or SR16.
  *   workspace: device scratch of at least mxfp4_linear_backward_workspace() bytes, 256-byte aligned;
  *   its contents are overwritten.  Calls sharing a workspace must be stream-ordered.
  *   Ordering: everything the call does is ordered after prior work of `cuda_stream` and before later work of it.

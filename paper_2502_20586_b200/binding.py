@@ -16,7 +16,7 @@ if not os.path.exists(LIB_PATH):
 _lib = C.CDLL(LIB_PATH)
 
 OK = 0
-ROUND_SR, ROUND_RN = 0, 1
+ROUND_SR, ROUND_RN, ROUND_SR16 = 0, 1, 2
 SF_LINEAR, SF_NATIVE = 0, 1
 OUT_BF16, OUT_FP32 = 0, 1
 

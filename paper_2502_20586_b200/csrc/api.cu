@@ -215,7 +215,7 @@ mxfp4_status mxfp4_rht_sr_quantize(const void* x, int64_t rows, int64_t cols, in
     if (codes == nullptr || scales == nullptr) return MXFP4_ERR_NULL;
     mxfp4_status st = check_quant(x, rows, cols, ld, reduce_dim, g);
     if (st != MXFP4_OK) return st;
-    if (rounding != MXFP4_ROUND_SR && rounding != MXFP4_ROUND_RN) return MXFP4_ERR_MODE;
+    if (rounding != MXFP4_ROUND_SR && rounding != MXFP4_ROUND_RN && rounding != MXFP4_ROUND_SR16) return MXFP4_ERR_MODE;
     if (sf_layout != MXFP4_SF_LINEAR && sf_layout != MXFP4_SF_NATIVE) return MXFP4_ERR_MODE;
     if (!aligned16(codes)) return MXFP4_ERR_ALIGN;
     if ((st = runtime_init()) != MXFP4_OK) return st;
@@ -267,7 +267,7 @@ mxfp4_status linear_backward_impl(const void* dY, const void* X, const void* W, 
     if (!valid_g(g)) return MXFP4_ERR_BAD_G;
     if (m % 128 != 0 || b % 128 != 0 || n % 8 != 0) return MXFP4_ERR_SHAPE;       // both reduce lengths feed the GEMM (K % 128)
     if (g != 0 && (m % g != 0 || b % g != 0)) return MXFP4_ERR_BAD_G;
-    if (rounding != MXFP4_ROUND_SR && rounding != MXFP4_ROUND_RN) return MXFP4_ERR_MODE;
+    if (rounding != MXFP4_ROUND_SR && rounding != MXFP4_ROUND_RN && rounding != MXFP4_ROUND_SR16) return MXFP4_ERR_MODE;
     if (out_dtype != MXFP4_OUT_BF16 && out_dtype != MXFP4_OUT_FP32) return MXFP4_ERR_MODE;
     if (accumulate != 0 && accumulate != 1) return MXFP4_ERR_MODE;
     if (accumulate == 1 && out_dtype != MXFP4_OUT_FP32) return MXFP4_ERR_MODE;      // accumulation is defined on fp32 gradients
@@ -301,7 +301,7 @@ mxfp4_status linear_backward_impl(const void* dY, const void* X, const void* W, 
             if (mx::launch_quantize(q[i], stream) != cudaSuccess) return MXFP4_ERR_CUDA;
     }
     // lines 7-11: two MXFP4 GEMMs; the 16/9 un-does the two 3/4 pre-scales of Algorithm 2.
-    const float alpha = rounding == MXFP4_ROUND_SR ? 16.0f / 9.0f : 1.0f;
+    const float alpha = rounding != MXFP4_ROUND_RN ? 16.0f / 9.0f : 1.0f;       // both SR modes carry the 3/4 pre-scale
     // Large problems (never the ones the fixed-scratch variant accepts) run the two GEMMs fork / join.
     const int64_t waves_dx = ((b + 255) / 256) * ((n + 255) / 256), waves_dw = ((m + 255) / 256) * ((n + 255) / 256);
     ForkJoin* fj = ws.total > (size_t)MXFP4_STATIC_WORKSPACE_BYTES && waves_dx >= 74 && waves_dw >= 74 ? fork_join() : nullptr;

@@ -11,7 +11,7 @@ struct QuantArgs {
     int64_t rows, cols, ld;
     int reduce_dim;       // 1: reduce along cols; 0: reduce along rows (transposed output)
     int g;                // 0, 32, 64, 128, 256
-    int rounding;         // 0 SR, 1 RN
+    int rounding;         // 0 SR, 1 RN, 2 SR with the 16-bit dither
     uint64_t seed;
     uint32_t stream_tag;
     uint8_t* codes;

@@ -148,6 +148,16 @@ __device__ __forceinline__ uint32_t cvt_f16x2_rz(float lo, float hi) {
     return d;
 }
 
+// cvt.rs.satfinite.e2m1x4.f32: four floats -> four E2M1 codes (v0 in the low nibble), rounded stochastically between
+// grid neighbours with a 16-bit dither per value taken from `rbits` (bytes b0..b3, low to high): round up iff
+// floor(65536 frac) + R >= 65536, where v0 uses R = 256 b2 + b0, v1 the same 16 bits reversed, v2 R = 256 b3 + b1 and
+// v3 that one reversed.  The sign is kept (a negative value may give -0), |v| >= 6 gives 6.
+__device__ __forceinline__ uint32_t cvt_e2m1x4_rs(float v0, float v1, float v2, float v3, uint32_t rbits) {
+    uint16_t d;
+    asm("cvt.rs.satfinite.e2m1x4.f32 %0, {%1, %2, %3, %4}, %5;" : "=h"(d) : "f"(v3), "f"(v2), "f"(v1), "f"(v0), "r"(rbits));
+    return d;
+}
+
 // (a & ~mask) | (b & mask) in one LOP3.
 __device__ __forceinline__ uint32_t bitselect(uint32_t a, uint32_t b, uint32_t mask) {
     uint32_t d;
@@ -176,6 +186,9 @@ __host__ __device__ inline PipeConsts make_pipe_consts() { return PipeConsts{8u,
 //     result leaves the finished 4-bit code s ccc in the top nibble of each lane, so eight codes are gathered
 //     with two byte permutes, one shift and one select.  Lanes pair elements (i, i+2) and (i+1, i+3), which is
 //     how the four draws of one Philox word split with one mask and one byte permute.
+//   SR16 (ROUNDING = 2; Algorithm 2 with a 16-bit dither): z = RZ(y * 3/4 * 2^-e) goes through the stochastic-rounding
+//     convert, four values and one Philox word at a time.  The truncation keeps floor(65536 frac) of the exact real
+//     because every threshold (a multiple of gap / 65536) is an fp32 number at that magnitude.
 //   RN (Algorithm 1): hardware nearest-even convert of y / X.
 // `rw` holds the block's 32 SR draws (sr_draws32); it is not read when ROUNDING = 1 (RN).
 // A NaN input is out of contract (the block's scale is then taken from the other values); Inf gives byte 255.
@@ -235,6 +248,19 @@ __device__ __forceinline__ void quantize_block32_rw(const float (&y)[32], const 
             const uint32_t od = __byte_perm(u[2], u[3], 0x7531);             // top bytes of elements 1, 3, 5, 7
             packed[q] = bitselect(ev >> 4, od, 0xF0F0F0F0u);
         }
+    } else if (ROUNDING == 2) {
+        if (scale_byte == 255u) {
+            packed[0] = packed[1] = packed[2] = packed[3] = 0u;
+            return;
+        }
+        const float c = 1.5f * pow2f_wide(-e - 1);                   // 3/4 * 2^-e; exact also where 2^(-e-1) is subnormal
+#pragma unroll
+        for (int q = 0; q < 4; ++q) {
+            const int i = 8 * q;
+            const uint32_t lo = cvt_e2m1x4_rs(__fmul_rz(y[i], c), __fmul_rz(y[i + 1], c), __fmul_rz(y[i + 2], c), __fmul_rz(y[i + 3], c), rw[2 * q]);
+            const uint32_t hi = cvt_e2m1x4_rs(__fmul_rz(y[i + 4], c), __fmul_rz(y[i + 5], c), __fmul_rz(y[i + 6], c), __fmul_rz(y[i + 7], c), rw[2 * q + 1]);
+            packed[q] = __byte_perm(lo, hi, 0x5410);
+        }
     } else {
         if (scale_byte == 255u) {
             packed[0] = packed[1] = packed[2] = packed[3] = 0u;
@@ -261,6 +287,9 @@ __device__ __forceinline__ void quantize_block32(const float (&y)[32], int round
     if (rounding == 0) {
         sr_draws32(seed, stream_tag, i0, rw);
         quantize_block32_rw<0>(y, rw, packed, scale_byte, make_pipe_consts());
+    } else if (rounding == 2) {
+        sr_draws32(seed, stream_tag, i0, rw);
+        quantize_block32_rw<2>(y, rw, packed, scale_byte, make_pipe_consts());
     } else {
         quantize_block32_rw<1>(y, rw, packed, scale_byte, make_pipe_consts());
     }

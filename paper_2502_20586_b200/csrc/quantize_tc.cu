@@ -127,7 +127,9 @@ __device__ __forceinline__ TilePos advance_tile(const QParams& p, const TilePos&
     return pos;
 }
 
-enum { kModeSR = 0, kModeRN = 1, kModeDump = 2 };
+enum { kModeSR = 0, kModeRN = 1, kModeDump = 2, kModeSR16 = 3 };
+constexpr bool mode_draws(int mode) { return mode == kModeSR || mode == kModeSR16; }
+constexpr int mode_rounding(int mode) { return mode == kModeSR16 ? 2 : mode; }        // template argument of quantize_block32_rw
 
 // KW = 128-wide k-tiles per entry of the tile list: 1, or 2 for g = 256 (a tile then spans one 256-chunk).
 template <int MODE, int KW>
@@ -276,7 +278,7 @@ quantize_tc_kernel(const __grid_constant__ QMaps maps, const __grid_constant__ Q
         uint32_t t = blockIdx.x + it * gridDim.x;
         TilePos pos = locate_tile(p, t < num_tiles ? t : 0u);
         uint32_t rw[8];
-        if (MODE == kModeSR) sr_draws32(p.keys, p.view[pos.v].stream_tag, first_elem(pos), rw);
+        if (mode_draws(MODE)) sr_draws32(p.keys, p.view[pos.v].stream_tag, first_elem(pos), rw);
         if (KW == 2) {
             // g = 256: a tile is one 256-chunk of 128 rows; its two k-tiles went through T_0 and T_1 into the accumulator
             // pair (b0, b0 + 1): u = A_lo T_0, v = A_hi T_1.  The transformed values are y[0..127] = u + v and
@@ -288,7 +290,7 @@ quantize_tc_kernel(const __grid_constant__ QMaps maps, const __grid_constant__ Q
             it = (uint32_t)pr;
             t = blockIdx.x + it * gridDim.x;
             pos = locate_tile(p, t < num_tiles ? t : 0u);
-            if (MODE == kModeSR) sr_draws32(p.keys, p.view[pos.v].stream_tag, first_elem(pos) + 128u * hh, rw);
+            if (mode_draws(MODE)) sr_draws32(p.keys, p.view[pos.v].stream_tag, first_elem(pos) + 128u * hh, rw);
             for (; t < num_tiles; t += stride2, it += 2) {
                 const int b0 = 2 * pr;
                 const QView& vw = p.view[pos.v];
@@ -332,7 +334,7 @@ quantize_tc_kernel(const __grid_constant__ QMaps maps, const __grid_constant__ Q
                         __syncwarp();
                         if (lane == 0) { mbar_arrive(&acc_empty[b0]); mbar_arrive(&acc_empty[b0 + 1]); }
                     }
-                    if (MODE == kModeSR) {
+                    if (mode_draws(MODE)) {
                         if (j < 3) sr_draws32(p.keys, tag_cur, i_cur + 32 * (j + 1), nx);
                         else sr_draws32(p.keys, tag_next, i_next, nx);
                     }
@@ -343,11 +345,11 @@ quantize_tc_kernel(const __grid_constant__ QMaps maps, const __grid_constant__ Q
                             for (int i = 0; i < 8; ++i) dst[i] = make_float4(y[4 * i], y[4 * i + 1], y[4 * i + 2], y[4 * i + 3]);
                         }
                     } else {
-                        quantize_block32_rw<MODE>(y, rw, packed, sb, p.pipe);
+                        quantize_block32_rw<mode_rounding(MODE)>(y, rw, packed, sb, p.pipe);
                         if (live) *reinterpret_cast<uint4*>(code_dst + 16 * j) = make_uint4(packed[0], packed[1], packed[2], packed[3]);
                         sb_all |= sb << (8 * j);
                     }
-                    if (MODE == kModeSR) {
+                    if (mode_draws(MODE)) {
 #pragma unroll
                         for (int i = 0; i < 8; ++i) rw[i] = nx[i];
                     }
@@ -390,7 +392,7 @@ quantize_tc_kernel(const __grid_constant__ QMaps maps, const __grid_constant__ Q
                     __syncwarp();
                     if (lane == 0) mbar_arrive(&acc_empty[b]);
                 }
-                if (MODE == kModeSR) {
+                if (mode_draws(MODE)) {
                     if (j < 3) sr_draws32(p.keys, tag_cur, i_cur + 32 * (j + 1), nx);
                     else sr_draws32(p.keys, tag_next, i_next, nx);
                 }
@@ -403,11 +405,11 @@ quantize_tc_kernel(const __grid_constant__ QMaps maps, const __grid_constant__ Q
                         for (int i = 0; i < 8; ++i) dst[i] = make_float4(y[4 * i], y[4 * i + 1], y[4 * i + 2], y[4 * i + 3]);
                     }
                 } else {
-                    quantize_block32_rw<MODE>(y, rw, packed, sb, p.pipe);
+                    quantize_block32_rw<mode_rounding(MODE)>(y, rw, packed, sb, p.pipe);
                     if (live) *reinterpret_cast<uint4*>(code_dst + 16 * j) = make_uint4(packed[0], packed[1], packed[2], packed[3]);
                     sb_all |= sb << (8 * j);
                 }
-                if (MODE == kModeSR) {
+                if (mode_draws(MODE)) {
 #pragma unroll
                     for (int i = 0; i < 8; ++i) rw[i] = nx[i];
                 }
@@ -442,9 +444,10 @@ bool quant_tc_eligible(const QuantArgs& a) {
 cudaError_t fetch_quant_tc_status(unsigned int* word) { return device_status_fetch(word); }
 
 cudaError_t quant_tc_init() {
-    const void* kernels[6] = {(const void*)quantize_tc_kernel<kModeSR, 1>, (const void*)quantize_tc_kernel<kModeRN, 1>,
-                              (const void*)quantize_tc_kernel<kModeDump, 1>, (const void*)quantize_tc_kernel<kModeSR, 2>,
-                              (const void*)quantize_tc_kernel<kModeRN, 2>, (const void*)quantize_tc_kernel<kModeDump, 2>};
+    const void* kernels[8] = {(const void*)quantize_tc_kernel<kModeSR, 1>, (const void*)quantize_tc_kernel<kModeRN, 1>,
+                              (const void*)quantize_tc_kernel<kModeDump, 1>, (const void*)quantize_tc_kernel<kModeSR16, 1>,
+                              (const void*)quantize_tc_kernel<kModeSR, 2>, (const void*)quantize_tc_kernel<kModeRN, 2>,
+                              (const void*)quantize_tc_kernel<kModeDump, 2>, (const void*)quantize_tc_kernel<kModeSR16, 2>};
     for (const void* k : kernels) {
         cudaError_t e = cudaFuncSetAttribute(k, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kSmemQ);
         if (e != cudaSuccess) return e;
@@ -506,6 +509,7 @@ cudaError_t launch_quantize_tc_group(const QuantArgs* a, int n, bool dump_y, cud
     void (*kernel)(QMaps, QParams);
     if (dump_y) kernel = wide ? quantize_tc_kernel<kModeDump, 2> : quantize_tc_kernel<kModeDump, 1>;
     else if (a[0].rounding == 0) kernel = wide ? quantize_tc_kernel<kModeSR, 2> : quantize_tc_kernel<kModeSR, 1>;
+    else if (a[0].rounding == 2) kernel = wide ? quantize_tc_kernel<kModeSR16, 2> : quantize_tc_kernel<kModeSR16, 1>;
     else kernel = wide ? quantize_tc_kernel<kModeRN, 2> : quantize_tc_kernel<kModeRN, 1>;
     cudaLaunchConfig_t cfg = {};
     cfg.gridDim = dim3(grid); cfg.blockDim = dim3(kThreadsQ); cfg.dynamicSmemBytes = kSmemQ; cfg.stream = stream;

@@ -59,6 +59,7 @@ def test_argument_validation_needs_no_device(lib):
     assert q(P, 64, 64, 64, 0, 128, 0, 0, 0, P, P, 1, 0) == 4
     assert q(P, 32, 64, 64, 2, 64, 0, 0, 0, P, P, 1, 0) == 5                      # reduce_dim
     assert q(P, 32, 64, 64, 1, 64, 7, 0, 0, P, P, 1, 0) == 5                      # rounding
+    assert q(P, 32, 64, 64, 1, 64, 3, 0, 0, P, P, 1, 0) == 5 and q(P, 32, 64, 64, 1, 64, -1, 0, 0, P, P, 1, 0) == 5
     assert q(P, 32, 64, 64, 1, 64, 0, 0, 0, P, P, 3, 0) == 5                      # layout
     assert q(P + 2, 32, 64, 64, 1, 64, 0, 0, 0, P, P, 1, 0) == 3                  # alignment
     assert q(P, 32, 64, 68, 1, 64, 0, 0, 0, P, P, 1, 0) == 3                      # ld % 8

@@ -24,10 +24,12 @@ def _bits(t):
 CASES = [("gpt_6p7b", "attn_out"), ("gpt_6p7b", "fc1"), ("gpt_6p7b", "qkv"), ("gpt_6p7b", "fc2"),
          ("gpt_1p3b", "qkv"), ("gpt_1p3b", "attn_out"), ("gpt_1p3b", "fc1"), ("gpt_1p3b", "fc2"),
          ("gpt_345m", "qkv"), ("gpt_345m", "attn_out"), ("gpt_345m", "fc1"), ("gpt_345m", "fc2")]
+# rounding mode per case: the 8-bit SR reading everywhere, the 16-bit one on the benchmark's layers and one small layer
+CASES = [c + (0,) for c in CASES] + [("gpt_6p7b", l, 2) for l in ("attn_out", "fc1", "qkv", "fc2")] + [("gpt_345m", "fc1", 2)]
 
 
-@pytest.mark.parametrize("config,layer_name", CASES)
-def test_sampled_parity_at_full_shapes(ref, config, layer_name):
+@pytest.mark.parametrize("config,layer_name,rounding", CASES)
+def test_sampled_parity_at_full_shapes(ref, config, layer_name, rounding):
     import torch
     if not torch.cuda.is_available():
         pytest.skip("no GPU")
@@ -52,14 +54,14 @@ def test_sampled_parity_at_full_shapes(ref, config, layer_name):
     }
     gpu_q, ora_q = {}, {}
     for tag, (t, rd, rows, host_rows) in views.items():
-        codes, scales = mx.mxfp4_rht_sr_quantize(t, rd, g, seed, tag, mx.ROUND_SR, mx.SF_NATIVE)
+        codes, scales = mx.mxfp4_rht_sr_quantize(t, rd, g, seed, tag, rounding, mx.SF_NATIVE)
         R, K = codes.shape[0], codes.shape[1] * 2
         rt = torch.from_numpy(rows).cuda()
         c = hp.unpack_codes(codes[rt, :].cpu().numpy())
         offs = torch.from_numpy(hp.sf_native_offsets(R, K)[rows, :]).cuda()
         s = scales[offs].cpu().numpy()
         gpu_q[tag] = (c, s, codes, scales)
-        _, oc, os_ = ref.rht_quantize(host_rows, g, ref.ROUND_SR, seed, tag, row_ids=rows)
+        _, oc, os_ = ref.rht_quantize(host_rows, g, rounding, seed, tag, row_ids=rows)
         ora_q[tag] = (oc, os_)
         same = (s == os_).repeat(32, axis=1)
         assert (s != os_).mean() <= 1e-4
@@ -81,7 +83,7 @@ def test_sampled_parity_at_full_shapes(ref, config, layer_name):
     del Cx, Cw
 
     # the one-call path, bf16 outputs as in the benchmark, against the oracle's own Algorithm 3 on the sampled rows
-    dX, dW = mx.mxfp4_linear_backward(dY, X, W, g, seed, mx.ROUND_SR, mx.OUT_BF16)
+    dX, dW = mx.mxfp4_linear_backward(dY, X, W, g, seed, rounding, mx.OUT_BF16)
     assert mx.mxfp4_device_status() == 0
     ox = ref.gemm(*ora_q[1], *ora_q[2], alpha=alpha); ow = ref.gemm(*ora_q[3], *ora_q[4], alpha=alpha)
     bx = dX[It][:, Jt].float().cpu().numpy().astype(np.float64); bw = dW[Pt][:, Qt].float().cpu().numpy().astype(np.float64)
