@@ -315,6 +315,23 @@ def run_gpu(args):
             ms_var = a.elapsed_time(b) / k_var
             variants[other] = {"ms_per_step": ms_var, "value": flops_step / (ms_var * 1e-3) / 1e12, "steps": k_var,
                                "note": "this rank's step with the other SR reading (8-bit centred dither / 16-bit dither of the hardware convert)"}
+        # the fused-producer variant (dY transformed and rounded inside the GEMM kernels), a few steps: it is several times slower
+        if g in (32, 64, 128) and all(l.b % 256 == 0 and l.m % 256 == 0 for l in layers):
+            def step_fused():
+                for (layer, dY, X, W, dX, dW) in data:
+                    mx.mxfp4_linear_backward_fused(dY, X, W, g, seed, rnd, out_dtype, dX=dX, dW=dW, workspace=ws)
+            step_fused()
+            a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            k_var = max(1, min(args.steps, 3))
+            barrier()
+            a.record(stream)
+            for _ in range(k_var):
+                step_fused()
+            b.record(stream)
+            barrier()
+            ms_var = a.elapsed_time(b) / k_var
+            variants["fused_producer"] = {"ms_per_step": ms_var, "value": flops_step / (ms_var * 1e-3) / 1e12, "steps": k_var,
+                                          "note": "Algorithm 3 with lines 3 and 5 inside the GEMM kernels: every 128 x 128 output tile re-quantises its A panel"}
 
     clocks = sampler.stop()
     if gemm_tflops is not None:

@@ -148,6 +148,35 @@ MXFP4_API mxfp4_status mxfp4_linear_backward_ex(const void* dY, const void* X, c
                                       void* workspace, size_t workspace_bytes, void* cuda_stream);
 
 /*
+ * Fused-producer variant (Section 3.2 proposes fusing the transform with the GEMM's operand path): a block-scaled
+ * FP4 GEMM whose A operand is transformed and quantised INSIDE the GEMM kernel, never written to global memory:
+ *     C[M, N] = alpha * Q(A blockdiag(S H_g / sqrt(g))) deq(B)^T
+ *   x, rows, cols, ld, reduce_dim, g, rounding, seed, stream_tag: as in mxfp4_rht_sr_quantize; A = x [M = rows,
+ *     K = cols] for reduce_dim 1, A = x^T [M = cols, K = rows] for reduce_dim 0.  g in {32, 64, 128}; K % 256 == 0.
+ *   B_codes [N, K/2], B_scales (NATIVE layout): the other operand, quantised beforehand.  N % 8 == 0.
+ *   C [M, N], leading dimension ldc, bf16 or fp32.
+ * The codes the kernel derives are those mxfp4_rht_sr_quantize would write for the same arguments (the SR draws are
+ * keyed on the element index), so the result equals mxfp4_gemm on that call's output.  Every CTA re-quantises the A
+ * panel of its 128 x 128 output tile, N / 128 times over the whole product: for wide N this is several times slower
+ * than quantising once and is offered for measurement and for narrow N.
+ * Errors as mxfp4_rht_sr_quantize and mxfp4_gemm; shapes the kernel does not take give MXFP4_ERR_SHAPE / BAD_G.
+ */
+MXFP4_API mxfp4_status mxfp4_gemm_fused(const void* x, int64_t rows, int64_t cols, int64_t ld, int reduce_dim,
+                                        int g, int rounding, uint64_t seed, uint32_t stream_tag,
+                                        const uint8_t* B_codes, const uint8_t* B_scales, int64_t N, float alpha,
+                                        void* C, int64_t ldc, int out_dtype, void* cuda_stream);
+
+/*
+ * Algorithm 3 on the fused-producer kernel: W^T and X^T (lines 4, 6) are quantised by the stand-alone kernel, dY and
+ * dY^T (lines 3, 5) inside the two GEMMs.  Arguments, workspace and results as mxfp4_linear_backward, with
+ * g in {32, 64, 128}, m % 256 == 0 and b % 256 == 0; codes, and therefore dX and dW, agree with that call's.
+ */
+MXFP4_API mxfp4_status mxfp4_linear_backward_fused(const void* dY, const void* X, const void* W,
+                                                   int64_t b, int64_t m, int64_t n, int g, int rounding, uint64_t seed,
+                                                   void* dX, void* dW, int out_dtype,
+                                                   void* workspace, size_t workspace_bytes, void* cuda_stream);
+
+/*
  * The same backward pass for callers that cannot supply a workspace.  (The paper has no counterpart: this is a
  * property of the library, not of the method.)
  *

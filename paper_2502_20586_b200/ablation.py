@@ -33,7 +33,7 @@ def mxfp4_product(A, B, g, rounding, seed, out=None):
     """quantise(A) quantise(B)^T through the C ABI; alpha = 16/9 with SR (Algorithm 3 lines 10-11)."""
     ca, sa = mx.mxfp4_rht_sr_quantize(A, 1, g, seed, 1, rounding, mx.SF_NATIVE)
     cb, sb = mx.mxfp4_rht_sr_quantize(B, 1, g, seed, 2, rounding, mx.SF_NATIVE)
-    return mx.mxfp4_gemm(ca, sa, cb, sb, 16.0 / 9.0 if rounding == mx.ROUND_SR else 1.0, mx.OUT_FP32, C_out=out)
+    return mx.mxfp4_gemm(ca, sa, cb, sb, 16.0 / 9.0 if rounding != mx.ROUND_RN else 1.0, mx.OUT_FP32, C_out=out)
 
 
 MODES = (("RHT+SR", True, mx.ROUND_SR), ("SR", False, mx.ROUND_SR), ("RHT+RN", True, mx.ROUND_RN), ("RN", False, mx.ROUND_RN))

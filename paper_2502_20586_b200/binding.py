@@ -37,6 +37,10 @@ _lib.mxfp4_linear_backward_ex_workspace.argtypes = [_i64, _i64, _i64, _int]
 _lib.mxfp4_linear_backward_ex_workspace.restype = _sz
 _lib.mxfp4_linear_backward_ex.argtypes = [_vp, _vp, _vp, _i64, _i64, _i64, _int, _int, _u64, _vp, _vp, _vp, _int, _int, _vp, _sz, _vp]
 _lib.mxfp4_linear_backward_ex.restype = _int
+_lib.mxfp4_gemm_fused.argtypes = [_vp, _i64, _i64, _i64, _int, _int, _int, _u64, _u32, _vp, _vp, _i64, C.c_float, _vp, _i64, _int, _vp]
+_lib.mxfp4_gemm_fused.restype = _int
+_lib.mxfp4_linear_backward_fused.argtypes = [_vp, _vp, _vp, _i64, _i64, _i64, _int, _int, _u64, _vp, _vp, _int, _vp, _sz, _vp]
+_lib.mxfp4_linear_backward_fused.restype = _int
 _lib.mxfp4_fp4_ceiling.argtypes = [_i64, C.POINTER(C.c_int64), _vp]
 _lib.mxfp4_fp4_ceiling.restype = _int
 _lib.mxfp4_scale_bytes.argtypes = [_i64, _i64, _int]
@@ -48,7 +52,8 @@ _lib.mxfp4_status_string.restype = C.c_char_p
 
 EXPORTS = ["mxfp4_rht_sr_quantize", "mxfp4_rht", "mxfp4_gemm", "mxfp4_linear_backward_workspace",
            "mxfp4_linear_backward", "mxfp4_linear_backward_static", "mxfp4_scale_bytes", "mxfp4_device_status", "mxfp4_status_string",
-           "mxfp4_fp4_ceiling", "mxfp4_linear_backward_ex_workspace", "mxfp4_linear_backward_ex"]
+           "mxfp4_fp4_ceiling", "mxfp4_linear_backward_ex_workspace", "mxfp4_linear_backward_ex", "mxfp4_gemm_fused",
+           "mxfp4_linear_backward_fused"]
 
 
 class MxFp4Error(RuntimeError):
@@ -115,6 +120,39 @@ def mxfp4_gemm(A_codes, A_scales, B_codes, B_scales, alpha: float = 1.0, out_dty
     _check(_lib.mxfp4_gemm(_ptr(A_codes), _ptr(A_scales), _ptr(B_codes), _ptr(B_scales), M, N, 2 * K2, SF_NATIVE,
                            alpha, _ptr(C_out), C_out.stride(0), out_dtype, _stream()))
     return C_out
+
+
+def mxfp4_gemm_fused(x, reduce_dim: int, g: int, seed: int, stream_tag: int, rounding: int, B_codes, B_scales,
+                     alpha: float = 1.0, out_dtype: int = OUT_BF16, C_out=None):
+    """C = alpha * Q(RHT(A)) deq(B)^T with A = x (reduce_dim 1) or x^T (reduce_dim 0) quantised inside the GEMM kernel."""
+    assert x.is_cuda and x.dtype == torch.bfloat16 and x.dim() == 2 and x.stride(1) == 1
+    rows, cols = x.shape
+    M = rows if reduce_dim == 1 else cols
+    N = B_codes.shape[0]
+    if C_out is None:
+        C_out = torch.empty((M, N), dtype=torch.float32 if out_dtype == OUT_FP32 else torch.bfloat16, device=x.device)
+    _check(_lib.mxfp4_gemm_fused(_ptr(x), rows, cols, x.stride(0), reduce_dim, g, rounding, seed, stream_tag, _ptr(B_codes),
+                                 _ptr(B_scales), N, alpha, _ptr(C_out), C_out.stride(0), out_dtype, _stream()))
+    return C_out
+
+
+def mxfp4_linear_backward_fused(dY, X, W, g: int, seed: int, rounding: int = ROUND_SR, out_dtype: int = OUT_BF16,
+                                dX=None, dW=None, workspace=None):
+    """Algorithm 3 with dY / dY^T transformed and quantised inside the two GEMM kernels (fused-producer variant)."""
+    b, m = dY.shape
+    _, n = X.shape
+    for t in (dY, X, W):
+        assert t.is_cuda and t.dtype == torch.bfloat16 and t.is_contiguous()
+    dt = torch.float32 if out_dtype == OUT_FP32 else torch.bfloat16
+    if dX is None:
+        dX = torch.empty((b, n), dtype=dt, device=dY.device)
+    if dW is None:
+        dW = torch.empty((m, n), dtype=dt, device=dY.device)
+    if workspace is None:
+        workspace = torch.empty(mxfp4_linear_backward_workspace(b, m, n), dtype=torch.uint8, device=dY.device)
+    _check(_lib.mxfp4_linear_backward_fused(_ptr(dY), _ptr(X), _ptr(W), b, m, n, g, rounding, seed, _ptr(dX), _ptr(dW),
+                                            out_dtype, _ptr(workspace), workspace.numel(), _stream()))
+    return dX, dW
 
 
 def mxfp4_linear_backward_workspace(b: int, m: int, n: int) -> int:

@@ -47,7 +47,9 @@ mxfp4_status runtime_init() {
             return;
         }
         g_rt.encode = reinterpret_cast<EncodeTiledFn>(fn);
-        if (mx::gemm_init() != cudaSuccess || mx::gemm_pair_init() != cudaSuccess || mx::quant_tc_init() != cudaSuccess) g_rt.status = MXFP4_ERR_CUDA;
+        if (mx::gemm_init() != cudaSuccess || mx::gemm_pair_init() != cudaSuccess || mx::quant_tc_init() != cudaSuccess ||
+            mx::gemm_fused_init() != cudaSuccess)
+            g_rt.status = MXFP4_ERR_CUDA;
         const char* pair = getenv("MXFP4_GEMM_PAIR");
         g_rt.gemm_pair = !(pair != nullptr && pair[0] == '0');
     });
@@ -169,6 +171,23 @@ mxfp4_status gemm_impl(const uint8_t* A_codes, const uint8_t* A_scales, const ui
     return mx::launch_gemm(a, stream) == cudaSuccess ? MXFP4_OK : MXFP4_ERR_CUDA;
 }
 
+// C = alpha Q(RHT(A)) deq(B)^T with A = x (reduce_dim 1) or x^T (reduce_dim 0) quantised inside the GEMM kernel.
+mxfp4_status gemm_fused_impl(const void* x, int64_t rows, int64_t cols, int64_t ld, int reduce_dim, int g, int rounding, uint64_t seed,
+                             uint32_t stream_tag, const uint8_t* B_codes, const uint8_t* B_scales, int64_t N, float alpha, void* C,
+                             int64_t ldc, int out_dtype, cudaStream_t stream) {
+    QuantArgs q{x, rows, cols, ld, reduce_dim, g, rounding, seed, stream_tag, nullptr, nullptr, 1, nullptr};
+    attach_input_map(q);
+    mx::FusedGemmArgs a;
+    a.tmap_x = q.tmap_x; a.has_tmap_x = q.has_tmap;
+    a.M = reduce_dim == 1 ? rows : cols; a.K = reduce_dim == 1 ? cols : rows; a.N = N;
+    a.sfb = B_scales; a.alpha = alpha; a.C = C; a.ldc = ldc; a.out_fp32 = out_dtype == MXFP4_OUT_FP32;
+    a.g = g; a.reduce_dim = reduce_dim; a.rounding = rounding; a.seed = seed; a.stream_tag = stream_tag;
+    if (!mx::gemm_fused_eligible(a)) return MXFP4_ERR_SHAPE;
+    const mxfp4_status st = make_codes_map(&a.tmap_b, B_codes, N, a.K, 128);
+    if (st != MXFP4_OK) return st;
+    return mx::launch_gemm_fused(a, stream) == cudaSuccess ? MXFP4_OK : MXFP4_ERR_CUDA;
+}
+
 struct Workspace {
     size_t codes[4], scales[4], total;
 };
@@ -248,6 +267,23 @@ mxfp4_status mxfp4_gemm(const uint8_t* A_codes, const uint8_t* A_scales, const u
     const mxfp4_status st = runtime_init();
     if (st != MXFP4_OK) return st;
     return gemm_impl(A_codes, A_scales, B_codes, B_scales, M, N, K, alpha, C, ldc, out_dtype, static_cast<cudaStream_t>(cuda_stream));
+}
+
+mxfp4_status mxfp4_gemm_fused(const void* x, int64_t rows, int64_t cols, int64_t ld, int reduce_dim, int g, int rounding, uint64_t seed,
+                              uint32_t stream_tag, const uint8_t* B_codes, const uint8_t* B_scales, int64_t N, float alpha, void* C,
+                              int64_t ldc, int out_dtype, void* cuda_stream) {
+    if (!B_codes || !B_scales || !C) return MXFP4_ERR_NULL;
+    mxfp4_status st = check_quant(x, rows, cols, ld, reduce_dim, g);
+    if (st != MXFP4_OK) return st;
+    if (g != 32 && g != 64 && g != 128) return MXFP4_ERR_BAD_G;
+    if (rounding != MXFP4_ROUND_SR && rounding != MXFP4_ROUND_RN && rounding != MXFP4_ROUND_SR16) return MXFP4_ERR_MODE;
+    if (out_dtype != MXFP4_OUT_BF16 && out_dtype != MXFP4_OUT_FP32) return MXFP4_ERR_MODE;
+    const int64_t K = reduce_dim == 1 ? cols : rows;
+    if (N <= 0 || N % 8 != 0 || ldc < N || K % 256 != 0 || N > 0x7FFFFFFF || rows > 0x7FFFFFFF || cols > 0x7FFFFFFF) return MXFP4_ERR_SHAPE;
+    if (!aligned16(B_codes) || !aligned16(B_scales) || !aligned16(C) || ldc % (out_dtype == MXFP4_OUT_FP32 ? 4 : 8) != 0) return MXFP4_ERR_ALIGN;
+    if ((st = runtime_init()) != MXFP4_OK) return st;
+    return gemm_fused_impl(x, rows, cols, ld, reduce_dim, g, rounding, seed, stream_tag, B_codes, B_scales, N, alpha, C, ldc, out_dtype,
+                           static_cast<cudaStream_t>(cuda_stream));
 }
 
 size_t mxfp4_linear_backward_workspace(int64_t b, int64_t m, int64_t n) {
@@ -339,11 +375,44 @@ mxfp4_status mxfp4_linear_backward_ex(const void* dY, const void* X, const void*
     return linear_backward_impl(dY, X, W, b, m, n, g, rounding, seed, dX, dW, db, out_dtype, accumulate, workspace, workspace_bytes, cuda_stream);
 }
 
+mxfp4_status mxfp4_linear_backward_fused(const void* dY, const void* X, const void* W, int64_t b, int64_t m, int64_t n, int g, int rounding,
+                                         uint64_t seed, void* dX, void* dW, int out_dtype, void* workspace, size_t workspace_bytes,
+                                         void* cuda_stream) {
+    if (!dY || !X || !W || !dX || !dW) return MXFP4_ERR_NULL;
+    if (b <= 0 || m <= 0 || n <= 0) return MXFP4_ERR_SHAPE;
+    if (g != 32 && g != 64 && g != 128) return MXFP4_ERR_BAD_G;
+    if (m % 256 != 0 || b % 256 != 0 || n % 8 != 0) return MXFP4_ERR_SHAPE;          // the fused kernel steps K by 256
+    if (rounding != MXFP4_ROUND_SR && rounding != MXFP4_ROUND_RN && rounding != MXFP4_ROUND_SR16) return MXFP4_ERR_MODE;
+    if (out_dtype != MXFP4_OUT_BF16 && out_dtype != MXFP4_OUT_FP32) return MXFP4_ERR_MODE;
+    if (!aligned16(dY) || !aligned16(X) || !aligned16(W) || !aligned16(dX) || !aligned16(dW)) return MXFP4_ERR_ALIGN;
+    const Workspace ws = plan_workspace(b, m, n);
+    if (workspace == nullptr || workspace_bytes < ws.total || (reinterpret_cast<uintptr_t>(workspace) & 255u) != 0) return MXFP4_ERR_WORKSPACE;
+    mxfp4_status st = runtime_init();
+    if (st != MXFP4_OK) return st;
+    cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
+    uint8_t* base = static_cast<uint8_t*>(workspace);
+    // lines 4 and 6: the B operands (W^T, X^T) are quantised once by the stand-alone kernel
+    QuantArgs q[2] = {
+        {W, m, n, n, 0, g, rounding, seed, 2u, base + ws.codes[1], base + ws.scales[1], 1, nullptr},
+        {X, b, n, n, 0, g, rounding, seed, 4u, base + ws.codes[3], base + ws.scales[3], 1, nullptr},
+    };
+    for (int i = 0; i < 2; ++i) {
+        attach_input_map(q[i]);
+        if (!mx::quant_tc_eligible(q[i])) return MXFP4_ERR_SHAPE;
+    }
+    if (mx::launch_quantize_tc_group(q, 2, false, stream) != cudaSuccess) return MXFP4_ERR_CUDA;
+    const float alpha = rounding != MXFP4_ROUND_RN ? 16.0f / 9.0f : 1.0f;
+    // lines 3 + 7 and 5 + 8: dY is transformed and rounded inside the GEMMs (stream tags 1 and 3)
+    st = gemm_fused_impl(dY, b, m, m, 1, g, rounding, seed, 1u, q[0].codes, q[0].scales, n, alpha, dX, n, out_dtype, stream);
+    if (st != MXFP4_OK) return st;
+    return gemm_fused_impl(dY, b, m, m, 0, g, rounding, seed, 3u, q[1].codes, q[1].scales, n, alpha, dW, n, out_dtype, stream);
+}
+
 mxfp4_status mxfp4_device_status(void* cuda_stream) {
     if (cudaStreamSynchronize(static_cast<cudaStream_t>(cuda_stream)) != cudaSuccess) return MXFP4_ERR_CUDA;
     unsigned int word = 0;
     cudaError_t (*const fetch[])(unsigned int*) = {mx::fetch_gemm_status, mx::fetch_gemm_pair_status, mx::fetch_quant_tc_status,
-                                                   mx::fetch_fp4_ceiling_status};
+                                                   mx::fetch_fp4_ceiling_status, mx::fetch_gemm_fused_status};
     for (auto f : fetch) {
         unsigned int w = 0;
         if (f(&w) != cudaSuccess) return MXFP4_ERR_CUDA;

@@ -65,6 +65,28 @@ cudaError_t fetch_gemm_pair_status(unsigned int* word);
 cudaError_t fetch_quant_tc_status(unsigned int* word);
 cudaError_t fetch_fp4_ceiling_status(unsigned int* word);
 
+// GEMM with the RHT + quantiser of its A operand fused into the kernel (gemm_fused.cu): A = x or x^T in bf16.
+struct FusedGemmArgs {
+    CUtensorMap tmap_x;   // x as [rows, cols] bf16, box 64 cols x 128 rows, 128-byte swizzle
+    bool has_tmap_x;
+    CUtensorMap tmap_b;   // codes [N, K/2] bytes, box 128 B x 128 rows
+    const uint8_t* sfb;   // native scale layout
+    int64_t M, N, K;
+    float alpha;
+    void* C;
+    int64_t ldc;
+    int out_fp32;
+    int g;                // 32, 64, 128
+    int reduce_dim;       // 1: A = x; 0: A = x^T
+    int rounding;
+    uint64_t seed;
+    uint32_t stream_tag;
+};
+bool gemm_fused_eligible(const FusedGemmArgs& a);
+cudaError_t launch_gemm_fused(const FusedGemmArgs& a, cudaStream_t stream);
+cudaError_t gemm_fused_init();
+cudaError_t fetch_gemm_fused_status(unsigned int* word);
+
 cudaError_t launch_gemm(const GemmArgs& a, cudaStream_t stream);
 cudaError_t gemm_init();            // one-time: opt in to large dynamic shared memory
 cudaError_t launch_gemm_pair(const GemmArgs& a, cudaStream_t stream);

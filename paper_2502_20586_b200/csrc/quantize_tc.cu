@@ -77,22 +77,6 @@ struct QMaps {
     CUtensorMap x[kQuantMaxViews];
 };
 
-// bf16 entry (n, k) of the transform operand, stored N x K (K-major): T[k][n] = S_k H_g[k][n] inside a g-chunk.
-// g = 256 (Sylvester: H_256 = [[H_128, H_128], [H_128, -H_128]]): entry (n, k) of the half-transform h, T_h[k][n] =
-// S_{128 h + k} H_128[k][n] / 16; the epilogue combines u = A_lo T_0 and v = A_hi T_1 into u + v and u - v.
-__device__ __forceinline__ uint32_t transform_entry_256(int n, int k, const uint32_t (&sign)[4]) {
-    const uint32_t neg = ((sign[k >> 5] >> (k & 31)) ^ (uint32_t)__popc(k & n)) & 1u;
-    return 0x3D80u | (neg << 15);                                         // 1/16 = exact 1/sqrt(256)
-}
-
-__device__ __forceinline__ uint32_t transform_entry(int n, int k, int g, const uint32_t (&sign)[4]) {
-    if ((n ^ k) & ~(g - 1)) return 0u;                                   // different g-chunks
-    const int kk = k & (g - 1);
-    const uint32_t neg = ((sign[kk >> 5] >> (kk & 31)) ^ (uint32_t)__popc(k & n & (g - 1))) & 1u;
-    const uint32_t mag = g == 64 ? 0x3E00u : 0x3F80u;                    // 1/8 (exact 1/sqrt(64)) or 1
-    return mag | (neg << 15);
-}
-
 // Position of a tile in the launch's list: its view and its (row tile, k tile) there.  Tiles of a view with a
 // contiguous reduce dimension run along k first, the transposing ones along the output rows first, so that CTAs
 // working side by side read neighbouring 256-byte row segments of x.

@@ -47,6 +47,7 @@ def main(argv=None):
     ap.add_argument("--no-flush", action="store_true")
     ap.add_argument("--bias", action="store_true", help="backward: also the bias gradient (extended entry point)")
     ap.add_argument("--accumulate", action="store_true", help="backward: accumulate into fp32 dW / db")
+    ap.add_argument("--fused", action="store_true", help="backward: the fused-producer variant (dY quantised inside the GEMM kernels)")
     args = ap.parse_args(argv)
     dev = torch.device("cuda", 0)
     torch.cuda.set_device(dev)
@@ -87,6 +88,9 @@ def main(argv=None):
             ws = torch.empty(mx.mxfp4_linear_backward_ex_workspace(b, m, n, args.bias), dtype=torch.uint8, device=dev)
             fn = lambda: mx.mxfp4_linear_backward_ex(dY, X, W, g, 0, args.rounding, out_dtype, dX=dX, dW=dW, db=db,
                                                      accumulate=args.accumulate, workspace=ws)
+        elif args.fused:
+            ws = torch.empty(mx.mxfp4_linear_backward_workspace(b, m, n), dtype=torch.uint8, device=dev)
+            fn = lambda: mx.mxfp4_linear_backward_fused(dY, X, W, g, 0, args.rounding, out_dtype, dX=dX, dW=dW, workspace=ws)
         else:
             ws = torch.empty(mx.mxfp4_linear_backward_workspace(b, m, n), dtype=torch.uint8, device=dev)
             fn = lambda: mx.mxfp4_linear_backward(dY, X, W, g, 0, args.rounding, out_dtype, dX=dX, dW=dW, workspace=ws)

@@ -91,6 +91,23 @@ def test_argument_validation_needs_no_device(lib):
     assert need0 == raw.mxfp4_linear_backward_workspace(256, 512, 512) and need1 > need0 and need1 % 256 == 0
     assert ex(P, P, P, 256, 512, 512, 64, 0, 0, P, P, P, 1, 0, P, need0, 0) == 6       # the bias scratch is missing
     assert raw.mxfp4_linear_backward_ex_workspace(256, 0, 512, 1) == 0
+    # fused-producer variant
+    gf = raw.mxfp4_gemm_fused
+    #      x  rows cols ld  rd g   rnd seed tag Bc Bs N    alpha C  ldc out stream
+    assert gf(P, 256, 512, 512, 1, 64, 0, 0, 1, 0, P, 128, 1.0, P, 128, 0, 0) == 1          # B codes NULL
+    assert gf(P, 256, 512, 512, 1, 256, 0, 0, 1, P, P, 128, 1.0, P, 128, 0, 0) == 4         # g = 256 is not taken
+    assert gf(P, 256, 512, 512, 1, 0, 0, 0, 1, P, P, 128, 1.0, P, 128, 0, 0) == 4           # nor g = 0
+    assert gf(P, 256, 384, 384, 1, 64, 0, 0, 1, P, P, 128, 1.0, P, 128, 0, 0) == 2          # K % 256
+    assert gf(P, 384, 256, 256, 0, 64, 0, 0, 1, P, P, 128, 1.0, P, 128, 0, 0) == 2          # K = rows for reduce_dim 0
+    assert gf(P, 256, 512, 512, 1, 64, 0, 0, 1, P, P, 100, 1.0, P, 128, 0, 0) == 2          # N % 8
+    assert gf(P, 256, 512, 512, 1, 64, 0, 0, 1, P, P, 128, 1.0, P, 64, 0, 0) == 2           # ldc < N
+    assert gf(P, 256, 512, 512, 1, 64, 5, 0, 1, P, P, 128, 1.0, P, 128, 0, 0) == 5          # rounding
+    assert gf(P, 256, 512, 512, 1, 64, 0, 0, 1, P, P + 8, 128, 1.0, P, 128, 0, 0) == 3      # alignment
+    lf = raw.mxfp4_linear_backward_fused
+    assert lf(P, P, P, 256, 512, 512, 256, 0, 0, P, P, 0, P, big, 0) == 4
+    assert lf(P, P, P, 256, 384, 512, 64, 0, 0, P, P, 0, P, big, 0) == 2                    # m % 256
+    assert lf(P, P, P, 256, 512, 512, 64, 0, 0, P, P, 0, P, 1024, 0) == 6
+    assert lf(P, P, P, 256, 512, 512, 64, 0, 0, 0, P, 0, P, big, 0) == 1
     # measurement aid
     assert raw.mxfp4_fp4_ceiling(0, C.byref(C.c_int64(0)), 0) == 2
     assert raw.mxfp4_fp4_ceiling(64, None, 0) == 2
