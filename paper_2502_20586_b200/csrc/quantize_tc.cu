@@ -113,7 +113,8 @@ __device__ __forceinline__ TilePos advance_tile(const QParams& p, const TilePos&
 
 enum { kModeSR = 0, kModeRN = 1, kModeDump = 2, kModeSR16 = 3 };
 constexpr bool mode_draws(int mode) { return mode == kModeSR || mode == kModeSR16; }
-constexpr int mode_rounding(int mode) { return mode == kModeSR16 ? 2 : mode; }        // template argument of quantize_block32_rw
+// template argument of quantize_block32_rw; the g = 256 kernel (kw = 2) rounds SR through the convert instruction (same codes, fewer registers)
+constexpr int mode_rounding(int mode, int kw) { return mode == kModeSR16 ? 2 : (mode == kModeSR && kw == 2) ? 3 : mode; }
 
 // KW = 128-wide k-tiles per entry of the tile list: 1, or 2 for g = 256 (a tile then spans one 256-chunk).
 template <int MODE, int KW>
@@ -329,7 +330,7 @@ quantize_tc_kernel(const __grid_constant__ QMaps maps, const __grid_constant__ Q
                             for (int i = 0; i < 8; ++i) dst[i] = make_float4(y[4 * i], y[4 * i + 1], y[4 * i + 2], y[4 * i + 3]);
                         }
                     } else {
-                        quantize_block32_rw<mode_rounding(MODE)>(y, rw, packed, sb, p.pipe);
+                        quantize_block32_rw<mode_rounding(MODE, KW)>(y, rw, packed, sb, p.pipe);
                         if (live) *reinterpret_cast<uint4*>(code_dst + 16 * j) = make_uint4(packed[0], packed[1], packed[2], packed[3]);
                         sb_all |= sb << (8 * j);
                     }
@@ -389,7 +390,7 @@ quantize_tc_kernel(const __grid_constant__ QMaps maps, const __grid_constant__ Q
                         for (int i = 0; i < 8; ++i) dst[i] = make_float4(y[4 * i], y[4 * i + 1], y[4 * i + 2], y[4 * i + 3]);
                     }
                 } else {
-                    quantize_block32_rw<mode_rounding(MODE)>(y, rw, packed, sb, p.pipe);
+                    quantize_block32_rw<mode_rounding(MODE, KW)>(y, rw, packed, sb, p.pipe);
                     if (live) *reinterpret_cast<uint4*>(code_dst + 16 * j) = make_uint4(packed[0], packed[1], packed[2], packed[3]);
                     sb_all |= sb << (8 * j);
                 }
