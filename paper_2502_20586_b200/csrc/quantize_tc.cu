@@ -382,7 +382,11 @@ quantize_tc_kernel(const __grid_constant__ QMaps maps, const __grid_constant__ Q
                     else sr_draws32(p.keys, tag_next, i_next, nx);
                 }
 #pragma unroll
-                for (int i = 0; i < 32; ++i) y[i] = __uint_as_float(raw[i]) * cg;   // exact no-op unless g is 32 or 128
+                for (int i = 0; i < 32; ++i) y[i] = __uint_as_float(raw[i]);
+                if (cg != 1.0f) {                               // g = 32, 128: 1/sqrt(g) is not a power of two (for g = 64 it is folded into T)
+#pragma unroll
+                    for (int i = 0; i < 32; ++i) y[i] *= cg;
+                }
                 if (MODE == kModeDump) {
                     if (live) {
                         float4* dst = reinterpret_cast<float4*>(y_dst + 32 * j);
