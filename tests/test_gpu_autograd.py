@@ -60,3 +60,48 @@ def test_seeds_advance_and_the_mean_gradient_converges(torch_gpu):
     mean_err = float((acc / T - dw_ref).norm() / dw_ref.norm())
     assert layer.calls == T
     assert mean_err < first / 4          # ideal: first / 8
+
+
+@pytest.mark.parametrize("rounding", ["SR", "SR16"])
+def test_a_small_network_trains_like_its_bf16_twin(torch_gpu, rounding):
+    """The recipe of Section 4 in miniature: bf16 forward, Algorithm-3 backward, fp32 master weights.  A two-layer
+    network fitted to a random teacher reaches the loss of the same network trained with exact bf16 gradients
+    (unbiased gradients with bounded variance only add noise that averages out over steps)."""
+    torch = torch_gpu
+    from paper_2502_20586_b200 import binding as mx
+    from paper_2502_20586_b200.autograd import MxFp4LinearFunction
+    gen = torch.Generator(device="cuda").manual_seed(9)
+    d_in, d_h, d_out, tokens = 256, 512, 256, 1024
+    teacher = torch.randn(d_in, d_out, device="cuda", generator=gen) / d_in ** 0.5
+    rnd = getattr(mx, "ROUND_" + rounding)
+
+    def run(mxfp4: bool):
+        g2 = torch.Generator(device="cuda").manual_seed(1)
+        w1 = (torch.randn(d_h, d_in, device="cuda", generator=g2) * 0.05).requires_grad_(True)      # fp32 master weights
+        w2 = (torch.randn(d_out, d_h, device="cuda", generator=g2) * 0.05).requires_grad_(True)
+        opt = torch.optim.SGD([w1, w2], lr=0.5, momentum=0.9)
+        data = torch.Generator(device="cuda").manual_seed(2)
+        losses = []
+        for step in range(120):
+            x = torch.randn(tokens, d_in, device="cuda", generator=data)
+            target = x @ teacher
+            xb = x.to(torch.bfloat16)
+            if mxfp4:
+                h = MxFp4LinearFunction.apply(xb, w1.to(torch.bfloat16), None, 64, 1000 + 2 * step, rnd)
+                y = MxFp4LinearFunction.apply(torch.relu(h), w2.to(torch.bfloat16), None, 64, 1001 + 2 * step, rnd)
+            else:
+                y = torch.relu(xb @ w1.to(torch.bfloat16).t()) @ w2.to(torch.bfloat16).t()
+            loss = ((y.float() - target) ** 2).mean()
+            opt.zero_grad()
+            loss.backward()
+            opt.step()
+            losses.append(float(loss.detach()))
+        return losses
+
+    ref = run(False)
+    ours = run(True)
+    assert mx.mxfp4_device_status() == 0
+    assert ref[-1] < 0.2 * ref[0]                                    # the task is learnable in 120 steps
+    tail_ref, tail_ours = np.mean(ref[-10:]), np.mean(ours[-10:])
+    assert tail_ours < 0.2 * ours[0]
+    assert tail_ours < 1.25 * tail_ref                         # close to the exact-gradient run
