@@ -239,18 +239,12 @@ def run_gpu(args):
     variants = {}
     fp4_peak = BF16_TO_FP4 * peaks["bf16_sustained"]
     if "roofline" in legs:
-        # ---- roofline: the same step as its six C-ABI calls per layer, CUDA events around each
-        # operand views of Algorithm 3: (tensor index in (dY, X, W), reduce_dim, stream tag)
-        views = ((0, 1, 1), (2, 0, 2), (0, 0, 3), (1, 0, 4))
+        # ---- roofline: the same step as its three launches per layer (one call that quantises the four operand views,
+        # two GEMM calls), CUDA events around each.  Quantiser bytes: bf16 read + codes and scales written, per element.
         bufs = []
         for (layer, dY, X, W, dX, dW) in data:
-            ops = []
-            for (ti, rd, tag) in views:
-                t = (dY, X, W)[ti]
-                R, K = (t.shape[0], t.shape[1]) if rd == 1 else (t.shape[1], t.shape[0])
-                ops.append((t, rd, tag, torch.empty((R, K // 2), dtype=torch.uint8, device=dev),
-                            torch.empty(mx.mxfp4_scale_bytes(R, K), dtype=torch.uint8, device=dev)))
-            bufs.append(ops)
+            wsl = torch.empty(mx.mxfp4_linear_backward_workspace(layer.b, layer.m, layer.n), dtype=torch.uint8, device=dev)
+            bufs.append((wsl, mx.mxfp4_quantize_operands(dY, X, W, g, seed, rnd, workspace=wsl)))
         records = []   # (kind, layer name, start event, end event, work)
 
         def timed(kind, name, work, fn):
@@ -259,16 +253,14 @@ def run_gpu(args):
             records.append((kind, name, a, b, work))
 
         def step_calls(record):
-            for (layer, dY, X, W, dX, dW), ops in zip(data, bufs):
-                for (t, rd, tag, codes, scales) in ops:
-                    fn = lambda t=t, rd=rd, tag=tag, codes=codes, scales=scales: mx.mxfp4_rht_sr_quantize(
-                        t, rd, g, seed, tag, rnd, mx.SF_NATIVE, codes=codes, scales=scales)
-                    if record:
-                        timed("quant_row" if rd == 1 else "quant_tr", layer.name, t.numel() * QUANT_BYTES_PER_ELEM, fn)
-                    else:
-                        fn()
+            for (layer, dY, X, W, dX, dW), (wsl, ops) in zip(data, bufs):
+                fn = lambda dY=dY, X=X, W=W, wsl=wsl: mx.mxfp4_quantize_operands(dY, X, W, g, seed, rnd, workspace=wsl)
+                if record:
+                    timed("quant", layer.name, (2 * dY.numel() + X.numel() + W.numel()) * QUANT_BYTES_PER_ELEM, fn)
+                else:
+                    fn()
                 for (a, bb, out, fl) in ((0, 1, dX, 2 * layer.b * layer.n * layer.m), (2, 3, dW, 2 * layer.m * layer.n * layer.b)):
-                    fn = lambda a=a, bb=bb, out=out, ops=ops: mx.mxfp4_gemm(ops[a][3], ops[a][4], ops[bb][3], ops[bb][4],
+                    fn = lambda a=a, bb=bb, out=out, ops=ops: mx.mxfp4_gemm(ops[a][0], ops[a][1], ops[bb][0], ops[bb][1],
                                                                              16.0 / 9.0 if rnd != 1 else 1.0, out_dtype, C_out=out)
                     if record:
                         timed("gemm", layer.name, fl, fn)
@@ -290,15 +282,28 @@ def run_gpu(args):
                                   for l in layers)
         gemm_tflops = gemm_fl / gemm_t / 1e12
         kernels = {}
-        for kind in ("quant_row", "quant_tr"):
-            t_, by, n_ = agg[kind]
-            kernels[kind] = {"launches": n_, "avg_ms": t_ / n_ * 1e3, "GB/s": by / t_ / 1e9,
-                             "frac_of_hbm_peak": by / t_ / 1e9 / peaks["hbm_gbs"]}
+        t_, by, n_ = agg["quant"]
+        kernels["quant"] = {"launches": n_, "avg_ms": t_ / n_ * 1e3, "GB/s": by / t_ / 1e9,
+                            "frac_of_hbm_peak": by / t_ / 1e9 / peaks["hbm_gbs"],
+                            "what": "the four operand views of a layer in one launch (dY row-wise and transposed, W and X transposed)"}
         kernels["gemm"] = {"launches": gemm_n, "avg_ms": gemm_t / gemm_n * 1e3, "TFLOP/s": gemm_tflops,
                            "frac_of_4x_bf16_sustained": gemm_tflops / fp4_peak,
                            "frac_of_4x_bf16_burst": gemm_tflops / (BF16_TO_FP4 * peaks["bf16_burst"]),
                            "frac_of_nominal_9pf": gemm_tflops / NOMINAL_FP4_TFLOPS}
         calls_ms = sum(v[0] for v in agg.values()) / k_roof * 1e3
+    clocks = sampler.stop()
+    if gemm_tflops is not None:
+        # On-box ceiling of the FP4 tensor pipe (resident operands, no loads, no epilogue): ~25 ms burst, ~0.3 s sustained.
+        def ceiling(mma_per_pair):
+            a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            a.record(stream); fl = mx.mxfp4_fp4_ceiling(mma_per_pair); b.record(stream)
+            torch.cuda.synchronize()
+            return fl / (a.elapsed_time(b) * 1e-3) / 1e12
+        ceiling(32000)
+        ceil_burst, ceil_sust = ceiling(320000), ceiling(3200000)
+        kernels["fp4_ceiling"] = {"burst_TFLOP/s": ceil_burst, "sustained_TFLOP/s": ceil_sust,
+                                  "gemm_frac_of_burst": gemm_tflops / ceil_burst, "gemm_frac_of_sustained": gemm_tflops / ceil_sust,
+                                  "what": "back-to-back 256x256x64 pair MMAs on shared-memory-resident operands"}
         # the other stochastic-rounding reading, same step, a short run
         if args.rounding in ("sr", "sr16"):
             other = "sr16" if args.rounding == "sr" else "sr"
@@ -314,7 +319,7 @@ def run_gpu(args):
             barrier()
             ms_var = a.elapsed_time(b) / k_var
             variants[other] = {"ms_per_step": ms_var, "value": flops_step / (ms_var * 1e-3) / 1e12, "steps": k_var,
-                               "note": "this rank's step with the other SR reading (8-bit centred dither / 16-bit dither of the hardware convert)"}
+                               "note": "this rank's step with the other SR reading (8-bit centred dither / 16-bit dither of the hardware convert), timed after the other legs on a warmer board: compare runs with --rounding for a like-for-like number"}
         # the fused-producer variant (dY transformed and rounded inside the GEMM kernels), a few steps: it is several times slower
         if g in (32, 64, 128) and all(l.b % 256 == 0 and l.m % 256 == 0 for l in layers):
             def step_fused():
@@ -333,19 +338,6 @@ def run_gpu(args):
             variants["fused_producer"] = {"ms_per_step": ms_var, "value": flops_step / (ms_var * 1e-3) / 1e12, "steps": k_var,
                                           "note": "Algorithm 3 with lines 3 and 5 inside the GEMM kernels: every 128 x 128 output tile re-quantises its A panel"}
 
-    clocks = sampler.stop()
-    if gemm_tflops is not None:
-        # On-box ceiling of the FP4 tensor pipe (resident operands, no loads, no epilogue): ~25 ms burst, ~0.3 s sustained.
-        def ceiling(mma_per_pair):
-            a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-            a.record(stream); fl = mx.mxfp4_fp4_ceiling(mma_per_pair); b.record(stream)
-            torch.cuda.synchronize()
-            return fl / (a.elapsed_time(b) * 1e-3) / 1e12
-        ceiling(32000)
-        ceil_burst, ceil_sust = ceiling(320000), ceiling(3200000)
-        kernels["fp4_ceiling"] = {"burst_TFLOP/s": ceil_burst, "sustained_TFLOP/s": ceil_sust,
-                                  "gemm_frac_of_burst": gemm_tflops / ceil_burst, "gemm_frac_of_sustained": gemm_tflops / ceil_sust,
-                                  "what": "back-to-back 256x256x64 pair MMAs on shared-memory-resident operands"}
     ms_e2e, h2d, d2h = None, 0, 0
     if "e2e" in legs:
         # ---- e2e: host buffers, copies inside the timed region

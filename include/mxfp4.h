@@ -133,6 +133,19 @@ MXFP4_API mxfp4_status mxfp4_linear_backward(const void* dY, const void* X, cons
                                    void* workspace, size_t workspace_bytes, void* cuda_stream);
 
 /*
+ * Algorithm 3 lines 3-6 alone: the four operand views of one layer (stream tags 1..4: dY, W^T, dY^T, X^T), quantised
+ * in ONE launch into `workspace` at the offsets mxfp4_operand_layout reports; lines 7-11 are then two mxfp4_gemm calls
+ * (dX = alpha Q1 Q2^T with M = b, N = n, K = m; dW = alpha Q3 Q4^T with M = m, N = n, K = b).  This is what
+ * mxfp4_linear_backward does internally; the split form lets a caller time the parts, or keep Q2 (the weights) for
+ * several micro-batches that share a seed.  Arguments and errors as mxfp4_linear_backward.
+ *   offsets[2 i], offsets[2 i + 1]: byte offsets of the codes and of the scales (NATIVE layout) of view i + 1.
+ */
+MXFP4_API void mxfp4_operand_layout(int64_t b, int64_t m, int64_t n, size_t offsets[8]);
+MXFP4_API mxfp4_status mxfp4_quantize_operands(const void* dY, const void* X, const void* W,
+                                               int64_t b, int64_t m, int64_t n, int g, int rounding, uint64_t seed,
+                                               void* workspace, size_t workspace_bytes, void* cuda_stream);
+
+/*
  * Algorithm 3 with the two remaining pieces of a linear layer's backward (problem statement, Section 2:
  * dL/db = 1 dL/dy; micro-batch gradient accumulation):
  *   db:         NULL, or fp32 [m] (16-byte aligned): the bias gradient, column sums of dY in fp32 (not quantised).

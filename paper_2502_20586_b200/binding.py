@@ -41,6 +41,10 @@ _lib.mxfp4_gemm_fused.argtypes = [_vp, _i64, _i64, _i64, _int, _int, _int, _u64,
 _lib.mxfp4_gemm_fused.restype = _int
 _lib.mxfp4_linear_backward_fused.argtypes = [_vp, _vp, _vp, _i64, _i64, _i64, _int, _int, _u64, _vp, _vp, _int, _vp, _sz, _vp]
 _lib.mxfp4_linear_backward_fused.restype = _int
+_lib.mxfp4_operand_layout.argtypes = [_i64, _i64, _i64, C.POINTER(_sz)]
+_lib.mxfp4_operand_layout.restype = None
+_lib.mxfp4_quantize_operands.argtypes = [_vp, _vp, _vp, _i64, _i64, _i64, _int, _int, _u64, _vp, _sz, _vp]
+_lib.mxfp4_quantize_operands.restype = _int
 _lib.mxfp4_fp4_ceiling.argtypes = [_i64, C.POINTER(C.c_int64), _vp]
 _lib.mxfp4_fp4_ceiling.restype = _int
 _lib.mxfp4_scale_bytes.argtypes = [_i64, _i64, _int]
@@ -53,7 +57,7 @@ _lib.mxfp4_status_string.restype = C.c_char_p
 EXPORTS = ["mxfp4_rht_sr_quantize", "mxfp4_rht", "mxfp4_gemm", "mxfp4_linear_backward_workspace",
            "mxfp4_linear_backward", "mxfp4_linear_backward_static", "mxfp4_scale_bytes", "mxfp4_device_status", "mxfp4_status_string",
            "mxfp4_fp4_ceiling", "mxfp4_linear_backward_ex_workspace", "mxfp4_linear_backward_ex", "mxfp4_gemm_fused",
-           "mxfp4_linear_backward_fused"]
+           "mxfp4_linear_backward_fused", "mxfp4_operand_layout", "mxfp4_quantize_operands"]
 
 
 class MxFp4Error(RuntimeError):
@@ -153,6 +157,28 @@ def mxfp4_linear_backward_fused(dY, X, W, g: int, seed: int, rounding: int = ROU
     _check(_lib.mxfp4_linear_backward_fused(_ptr(dY), _ptr(X), _ptr(W), b, m, n, g, rounding, seed, _ptr(dX), _ptr(dW),
                                             out_dtype, _ptr(workspace), workspace.numel(), _stream()))
     return dX, dW
+
+
+def mxfp4_quantize_operands(dY, X, W, g: int, seed: int, rounding: int = ROUND_SR, workspace=None):
+    """Algorithm 3 lines 3-6 in one launch.  Returns [(codes, scales)] for Q1..Q4 as views into the workspace
+    (codes [R, K/2] u8, scales flat u8 in the native layout), ready for mxfp4_gemm."""
+    b, m = dY.shape
+    _, n = X.shape
+    for t in (dY, X, W):
+        assert t.is_cuda and t.dtype == torch.bfloat16 and t.is_contiguous()
+    if workspace is None:
+        workspace = torch.empty(mxfp4_linear_backward_workspace(b, m, n), dtype=torch.uint8, device=dY.device)
+    _check(_lib.mxfp4_quantize_operands(_ptr(dY), _ptr(X), _ptr(W), b, m, n, g, rounding, seed, _ptr(workspace), workspace.numel(),
+                                        _stream()))
+    off = (_sz * 8)()
+    _lib.mxfp4_operand_layout(b, m, n, off)
+    shapes = ((b, m), (n, m), (m, b), (n, b))
+    out = []
+    for i, (R, K) in enumerate(shapes):
+        codes = workspace[off[2 * i]: off[2 * i] + R * K // 2].view(R, K // 2)
+        scales = workspace[off[2 * i + 1]: off[2 * i + 1] + mxfp4_scale_bytes(R, K)]
+        out.append((codes, scales))
+    return out
 
 
 def mxfp4_linear_backward_workspace(b: int, m: int, n: int) -> int:

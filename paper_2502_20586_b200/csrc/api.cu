@@ -294,6 +294,39 @@ size_t mxfp4_linear_backward_workspace(int64_t b, int64_t m, int64_t n) {
 }  // extern "C"
 
 namespace {
+// Algorithm 3 lines 3-6: the four operand views, stream tags 1..4, one sign vector (same seed) for all of them.
+mxfp4_status quantize_operands_impl(const void* dY, const void* X, const void* W, int64_t b, int64_t m, int64_t n, int g, int rounding,
+                                    uint64_t seed, uint8_t* const c[4], uint8_t* const s[4], cudaStream_t stream) {
+    QuantArgs q[4] = {
+        {dY, b, m, m, 1, g, rounding, seed, 1u, c[0], s[0], 1, nullptr},   // dY   [b, K = m]
+        {W, m, n, n, 0, g, rounding, seed, 2u, c[1], s[1], 1, nullptr},    // W^T  [n, K = m]
+        {dY, b, m, m, 0, g, rounding, seed, 3u, c[2], s[2], 1, nullptr},   // dY^T [m, K = b]
+        {X, b, n, n, 0, g, rounding, seed, 4u, c[3], s[3], 1, nullptr},    // X^T  [n, K = b]
+    };
+    bool all_tc = true;
+    for (int i = 0; i < 4; ++i) {
+        attach_input_map(q[i]);
+        all_tc = all_tc && mx::quant_tc_eligible(q[i]);
+    }
+    if (all_tc)                                     // the four views of the call in one launch
+        return mx::launch_quantize_tc_group(q, 4, false, stream) == cudaSuccess ? MXFP4_OK : MXFP4_ERR_CUDA;
+    for (int i = 0; i < 4; ++i)
+        if (mx::launch_quantize(q[i], stream) != cudaSuccess) return MXFP4_ERR_CUDA;
+    return MXFP4_OK;
+}
+
+// Argument checks shared by the entry points that take a whole layer.
+mxfp4_status check_layer(const void* dY, const void* X, const void* W, int64_t b, int64_t m, int64_t n, int g, int rounding) {
+    if (!dY || !X || !W) return MXFP4_ERR_NULL;
+    if (b <= 0 || m <= 0 || n <= 0) return MXFP4_ERR_SHAPE;
+    if (!valid_g(g)) return MXFP4_ERR_BAD_G;
+    if (m % 128 != 0 || b % 128 != 0 || n % 8 != 0) return MXFP4_ERR_SHAPE;       // both reduce lengths feed the GEMM (K % 128)
+    if (g != 0 && (m % g != 0 || b % g != 0)) return MXFP4_ERR_BAD_G;
+    if (rounding != MXFP4_ROUND_SR && rounding != MXFP4_ROUND_RN && rounding != MXFP4_ROUND_SR16) return MXFP4_ERR_MODE;
+    if (!aligned16(dY) || !aligned16(X) || !aligned16(W)) return MXFP4_ERR_ALIGN;
+    return MXFP4_OK;
+}
+
 // Algorithm 3, optionally with the bias gradient (db != NULL) and accumulation into dW and db.
 mxfp4_status linear_backward_impl(const void* dY, const void* X, const void* W, int64_t b, int64_t m, int64_t n, int g, int rounding,
                                   uint64_t seed, void* dX, void* dW, float* db, int out_dtype, int accumulate, void* workspace,
@@ -318,24 +351,7 @@ mxfp4_status linear_backward_impl(const void* dY, const void* X, const void* W, 
     uint8_t* base = static_cast<uint8_t*>(workspace);
     uint8_t *c[4], *s[4];
     for (int i = 0; i < 4; ++i) { c[i] = base + ws.codes[i]; s[i] = base + ws.scales[i]; }
-    // Algorithm 3 lines 3-6: stream tags 1..4, one sign vector (same seed) for all four views.
-    QuantArgs q[4] = {
-        {dY, b, m, m, 1, g, rounding, seed, 1u, c[0], s[0], 1, nullptr},   // dY   [b, K = m]
-        {W, m, n, n, 0, g, rounding, seed, 2u, c[1], s[1], 1, nullptr},    // W^T  [n, K = m]
-        {dY, b, m, m, 0, g, rounding, seed, 3u, c[2], s[2], 1, nullptr},   // dY^T [m, K = b]
-        {X, b, n, n, 0, g, rounding, seed, 4u, c[3], s[3], 1, nullptr},    // X^T  [n, K = b]
-    };
-    bool all_tc = true;
-    for (int i = 0; i < 4; ++i) {
-        attach_input_map(q[i]);
-        all_tc = all_tc && mx::quant_tc_eligible(q[i]);
-    }
-    if (all_tc) {                                   // the four views of the call in one launch
-        if (mx::launch_quantize_tc_group(q, 4, false, stream) != cudaSuccess) return MXFP4_ERR_CUDA;
-    } else {
-        for (int i = 0; i < 4; ++i)
-            if (mx::launch_quantize(q[i], stream) != cudaSuccess) return MXFP4_ERR_CUDA;
-    }
+    if ((st = quantize_operands_impl(dY, X, W, b, m, n, g, rounding, seed, c, s, stream)) != MXFP4_OK) return st;
     // lines 7-11: two MXFP4 GEMMs; the 16/9 un-does the two 3/4 pre-scales of Algorithm 2.
     const float alpha = rounding != MXFP4_ROUND_RN ? 16.0f / 9.0f : 1.0f;       // both SR modes carry the 3/4 pre-scale
     // Large problems (never the ones the fixed-scratch variant accepts) run the two GEMMs fork / join.
@@ -406,6 +422,27 @@ mxfp4_status mxfp4_linear_backward_fused(const void* dY, const void* X, const vo
     st = gemm_fused_impl(dY, b, m, m, 1, g, rounding, seed, 1u, q[0].codes, q[0].scales, n, alpha, dX, n, out_dtype, stream);
     if (st != MXFP4_OK) return st;
     return gemm_fused_impl(dY, b, m, m, 0, g, rounding, seed, 3u, q[1].codes, q[1].scales, n, alpha, dW, n, out_dtype, stream);
+}
+
+void mxfp4_operand_layout(int64_t b, int64_t m, int64_t n, size_t offsets[8]) {
+    if (offsets == nullptr) return;
+    for (int i = 0; i < 8; ++i) offsets[i] = 0;
+    if (b <= 0 || m <= 0 || n <= 0) return;
+    const Workspace ws = plan_workspace(b, m, n);
+    for (int i = 0; i < 4; ++i) { offsets[2 * i] = ws.codes[i]; offsets[2 * i + 1] = ws.scales[i]; }
+}
+
+mxfp4_status mxfp4_quantize_operands(const void* dY, const void* X, const void* W, int64_t b, int64_t m, int64_t n, int g, int rounding,
+                                     uint64_t seed, void* workspace, size_t workspace_bytes, void* cuda_stream) {
+    mxfp4_status st = check_layer(dY, X, W, b, m, n, g, rounding);
+    if (st != MXFP4_OK) return st;
+    const Workspace ws = plan_workspace(b, m, n);
+    if (workspace == nullptr || workspace_bytes < ws.total || (reinterpret_cast<uintptr_t>(workspace) & 255u) != 0) return MXFP4_ERR_WORKSPACE;
+    if ((st = runtime_init()) != MXFP4_OK) return st;
+    uint8_t* base = static_cast<uint8_t*>(workspace);
+    uint8_t *c[4], *s[4];
+    for (int i = 0; i < 4; ++i) { c[i] = base + ws.codes[i]; s[i] = base + ws.scales[i]; }
+    return quantize_operands_impl(dY, X, W, b, m, n, g, rounding, seed, c, s, static_cast<cudaStream_t>(cuda_stream));
 }
 
 mxfp4_status mxfp4_device_status(void* cuda_stream) {

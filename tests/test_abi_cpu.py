@@ -108,6 +108,18 @@ def test_argument_validation_needs_no_device(lib):
     assert lf(P, P, P, 256, 384, 512, 64, 0, 0, P, P, 0, P, big, 0) == 2                    # m % 256
     assert lf(P, P, P, 256, 512, 512, 64, 0, 0, P, P, 0, P, 1024, 0) == 6
     assert lf(P, P, P, 256, 512, 512, 64, 0, 0, 0, P, 0, P, big, 0) == 1
+    # split form
+    qo = raw.mxfp4_quantize_operands
+    assert qo(P, P, 0, 256, 512, 512, 64, 0, 0, P, big, 0) == 1
+    assert qo(P, P, P, 256, 500, 512, 64, 0, 0, P, big, 0) == 2
+    assert qo(P, P, P, 256, 512, 512, 96, 0, 0, P, big, 0) == 4
+    assert qo(P, P, P, 256, 512, 512, 64, 9, 0, P, big, 0) == 5
+    assert qo(P, P, P, 256, 512, 512, 64, 0, 0, P, 1024, 0) == 6
+    off = (C.c_size_t * 8)()
+    raw.mxfp4_operand_layout(256, 512, 512, off)
+    assert list(off) == sorted(off) and off[0] == 0 and all(o % 1024 == 0 for o in off)
+    assert off[7] + lib.mxfp4_scale_bytes(512, 256) <= raw.mxfp4_linear_backward_workspace(256, 512, 512)
+    assert off[1] - off[0] >= 256 * 512 // 2 and off[2] - off[1] >= lib.mxfp4_scale_bytes(256, 512)
     # measurement aid
     assert raw.mxfp4_fp4_ceiling(0, C.byref(C.c_int64(0)), 0) == 2
     assert raw.mxfp4_fp4_ceiling(64, None, 0) == 2

@@ -348,3 +348,26 @@ def test_linear_backward_is_bitwise_reproducible(gpu):
     other = gpu.mxfp4_linear_backward_ex(dY, X, W, g, 22, gpu.ROUND_SR, gpu.OUT_FP32, with_bias=True)
     assert not torch.equal(first[0], other[0]) and torch.equal(first[2], other[2])      # the seed moves dX, not the bias sums
     assert gpu.mxfp4_device_status() == 0
+
+
+def test_split_form_equals_the_one_call_form(gpu):
+    """mxfp4_quantize_operands + two mxfp4_gemm calls give bit for bit what mxfp4_linear_backward gives."""
+    import torch
+    gen = torch.Generator(device="cuda").manual_seed(13)
+    b, m, n, g = 512, 384, 264, 128
+    dY = (torch.randn(b, m, device="cuda", generator=gen) * 1e-3).to(torch.bfloat16)
+    X = torch.randn(b, n, device="cuda", generator=gen).to(torch.bfloat16)
+    W = (torch.randn(m, n, device="cuda", generator=gen) * 0.02).to(torch.bfloat16)
+    for rounding, alpha in ((gpu.ROUND_SR, 16 / 9), (gpu.ROUND_RN, 1.0), (gpu.ROUND_SR16, 16 / 9)):
+        q = gpu.mxfp4_quantize_operands(dY, X, W, g, 17, rounding)
+        dX = gpu.mxfp4_gemm(q[0][0], q[0][1], q[1][0], q[1][1], alpha, gpu.OUT_FP32)
+        dW = gpu.mxfp4_gemm(q[2][0], q[2][1], q[3][0], q[3][1], alpha, gpu.OUT_FP32)
+        rX, rW = gpu.mxfp4_linear_backward(dY, X, W, g, 17, rounding, gpu.OUT_FP32)
+        assert torch.equal(dX, rX) and torch.equal(dW, rW)
+        # and each view equals the single-operand call with its stream tag
+        for i, (t, rd) in enumerate(((dY, 1), (W, 0), (dY, 0), (X, 0))):
+            c, s = gpu.mxfp4_rht_sr_quantize(t, rd, g, 17, i + 1, rounding, gpu.SF_NATIVE)
+            R, K = c.shape[0], 2 * c.shape[1]                 # padding bytes of the tiled scale layout are not written: compare the decoded scales
+            assert torch.equal(c, q[i][0])
+            assert np.array_equal(hp.sf_native_to_linear(s.cpu().numpy(), R, K), hp.sf_native_to_linear(q[i][1].cpu().numpy(), R, K))
+    assert gpu.mxfp4_device_status() == 0
