@@ -24,21 +24,17 @@ struct Runtime {
     mxfp4_status status = MXFP4_OK;
     EncodeTiledFn encode = nullptr;
     bool gemm_pair = true;       // CTA-pair GEMM (gemm_pair.cu); MXFP4_GEMM_PAIR=0 selects the 1-CTA kernel (gemm.cu)
+    std::mutex mu;
+    static constexpr int kMaxDevices = 64;
+    mxfp4_status dev_status[kMaxDevices];
+    bool dev_done[kMaxDevices] = {};
 };
 Runtime g_rt;
 
-// One-time set-up: device check, driver entry point for tensor-map encoding, shared-memory opt-in.
+// Set-up: once per process the driver entry point for tensor-map encoding and the environment switches; once per
+// device (kernel attributes belong to the device's context) the capability check and the shared-memory opt-in.
 mxfp4_status runtime_init() {
     std::call_once(g_rt.once, [] {
-        int dev = 0, major = 0;
-        if (cudaGetDevice(&dev) != cudaSuccess || cudaDeviceGetAttribute(&major, cudaDevAttrComputeCapabilityMajor, dev) != cudaSuccess) {
-            g_rt.status = MXFP4_ERR_CUDA;
-            return;
-        }
-        if (major != 10) {
-            g_rt.status = MXFP4_ERR_DEVICE;
-            return;
-        }
         void* fn = nullptr;
         cudaDriverEntryPointQueryResult qres;
         if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &fn, cudaEnableDefault, &qres) != cudaSuccess || fn == nullptr ||
@@ -47,13 +43,25 @@ mxfp4_status runtime_init() {
             return;
         }
         g_rt.encode = reinterpret_cast<EncodeTiledFn>(fn);
-        if (mx::gemm_init() != cudaSuccess || mx::gemm_pair_init() != cudaSuccess || mx::quant_tc_init() != cudaSuccess ||
-            mx::gemm_fused_init() != cudaSuccess)
-            g_rt.status = MXFP4_ERR_CUDA;
         const char* pair = getenv("MXFP4_GEMM_PAIR");
         g_rt.gemm_pair = !(pair != nullptr && pair[0] == '0');
     });
-    return g_rt.status;
+    if (g_rt.status != MXFP4_OK) return g_rt.status;
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= Runtime::kMaxDevices) return MXFP4_ERR_CUDA;
+    std::lock_guard<std::mutex> lock(g_rt.mu);
+    if (!g_rt.dev_done[dev]) {
+        int major = 0;
+        mxfp4_status st = MXFP4_OK;
+        if (cudaDeviceGetAttribute(&major, cudaDevAttrComputeCapabilityMajor, dev) != cudaSuccess) st = MXFP4_ERR_CUDA;
+        else if (major != 10) st = MXFP4_ERR_DEVICE;
+        else if (mx::gemm_init() != cudaSuccess || mx::gemm_pair_init() != cudaSuccess || mx::quant_tc_init() != cudaSuccess ||
+                 mx::gemm_fused_init() != cudaSuccess)
+            st = MXFP4_ERR_CUDA;
+        g_rt.dev_status[dev] = st;
+        g_rt.dev_done[dev] = true;
+    }
+    return g_rt.dev_status[dev];
 }
 
 // Side stream and events for running the two independent GEMMs of a backward call side by side (fork / join around
