@@ -79,7 +79,11 @@ class ClockSampler:
         for line in self.proc.stdout:
             self.rows.append([t.strip() for t in line.split(",")])
 
-    def stop(self):
+    def mark(self):
+        """Number of samples taken so far (to tell the timed region from the legs that follow it)."""
+        return len(self.rows)
+
+    def stop(self, n_timed=None):
         if self.proc is None:
             return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvidia-smi unavailable"]}
         self.proc.terminate()
@@ -102,8 +106,20 @@ class ClockSampler:
         # median over samples under load (at least half of the maximum power seen)
         busy = sorted(s for s, p in zip([float(r[0]) for r in self.rows if len(r) >= 7], power) if p >= 0.5 * max(power)) if power else []
         med = busy[len(busy) // 2] if busy else (sm[len(sm) // 2] if sm else None)
-        return {"sm_mhz": med, "sm_max_mhz": smax, "power_w_max": max(power) if power else None,
-                "samples": len(sm), "reasons": sorted(reasons)}
+        out = {"sm_mhz": med, "sm_max_mhz": smax, "power_w_max": max(power) if power else None,
+               "samples": len(sm), "reasons": sorted(reasons),
+               "what": "nvidia-smi samples over all GPU legs of this run; sm_mhz = median of the samples under load"}
+        if n_timed:
+            timed = []
+            for r in self.rows[:n_timed]:
+                try:
+                    timed.append(float(r[0]))
+                except (ValueError, IndexError):
+                    pass
+            timed.sort()
+            if timed:
+                out["timed_region"] = {"samples": len(timed), "sm_mhz_median": timed[len(timed) // 2], "sm_mhz_min": timed[0]}
+        return out
 
 
 # ------------------------------------------------------------------------------------------ reference arm
@@ -235,8 +251,8 @@ def run_gpu(args):
         raise RuntimeError("a device-side wait timed out during the timed region")
 
     legs = set(args.legs.split(","))
-    kernels, calls_ms, gemm_tflops, clocks = {}, None, None, None
-    variants = {}
+    n_timed = sampler.mark()                    # samples up to here cover the warm-up and the timed steps
+    kernels, calls_ms, gemm_tflops = {}, None, None
     fp4_peak = BF16_TO_FP4 * peaks["bf16_sustained"]
     if "roofline" in legs:
         # ---- roofline: the same step as its three launches per layer (one call that quantises the four operand views,
@@ -291,19 +307,8 @@ def run_gpu(args):
                            "frac_of_4x_bf16_burst": gemm_tflops / (BF16_TO_FP4 * peaks["bf16_burst"]),
                            "frac_of_nominal_9pf": gemm_tflops / NOMINAL_FP4_TFLOPS}
         calls_ms = sum(v[0] for v in agg.values()) / k_roof * 1e3
-    clocks = sampler.stop()
-    if gemm_tflops is not None:
-        # On-box ceiling of the FP4 tensor pipe (resident operands, no loads, no epilogue): ~25 ms burst, ~0.3 s sustained.
-        def ceiling(mma_per_pair):
-            a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-            a.record(stream); fl = mx.mxfp4_fp4_ceiling(mma_per_pair); b.record(stream)
-            torch.cuda.synchronize()
-            return fl / (a.elapsed_time(b) * 1e-3) / 1e12
-        ceiling(32000)
-        ceil_burst, ceil_sust = ceiling(320000), ceiling(3200000)
-        kernels["fp4_ceiling"] = {"burst_TFLOP/s": ceil_burst, "sustained_TFLOP/s": ceil_sust,
-                                  "gemm_frac_of_burst": gemm_tflops / ceil_burst, "gemm_frac_of_sustained": gemm_tflops / ceil_sust,
-                                  "what": "back-to-back 256x256x64 pair MMAs on shared-memory-resident operands"}
+    variants = {}
+    if "roofline" in legs:
         # the other stochastic-rounding reading, same step, a short run
         if args.rounding in ("sr", "sr16"):
             other = "sr16" if args.rounding == "sr" else "sr"
@@ -319,7 +324,7 @@ def run_gpu(args):
             barrier()
             ms_var = a.elapsed_time(b) / k_var
             variants[other] = {"ms_per_step": ms_var, "value": flops_step / (ms_var * 1e-3) / 1e12, "steps": k_var,
-                               "note": "this rank's step with the other SR reading (8-bit centred dither / 16-bit dither of the hardware convert), timed after the other legs on a warmer board: compare runs with --rounding for a like-for-like number"}
+                               "note": "this rank's step with the other SR reading (8-bit centred dither / 16-bit dither of the hardware convert), timed right after the main steps; compare runs with --rounding for a like-for-like number"}
         # the fused-producer variant (dY transformed and rounded inside the GEMM kernels), a few steps: it is several times slower
         if g in (32, 64, 128) and all(l.b % 256 == 0 and l.m % 256 == 0 for l in layers):
             def step_fused():
@@ -338,6 +343,19 @@ def run_gpu(args):
             variants["fused_producer"] = {"ms_per_step": ms_var, "value": flops_step / (ms_var * 1e-3) / 1e12, "steps": k_var,
                                           "note": "Algorithm 3 with lines 3 and 5 inside the GEMM kernels: every 128 x 128 output tile re-quantises its A panel"}
 
+    if gemm_tflops is not None:
+        # On-box ceiling of the FP4 tensor pipe (resident operands, no loads, no epilogue): ~25 ms burst, ~0.3 s sustained.
+        def ceiling(mma_per_pair):
+            a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            a.record(stream); fl = mx.mxfp4_fp4_ceiling(mma_per_pair); b.record(stream)
+            torch.cuda.synchronize()
+            return fl / (a.elapsed_time(b) * 1e-3) / 1e12
+        ceiling(32000)
+        ceil_burst, ceil_sust = ceiling(320000), ceiling(3200000)
+        kernels["fp4_ceiling"] = {"burst_TFLOP/s": ceil_burst, "sustained_TFLOP/s": ceil_sust,
+                                  "gemm_frac_of_burst": gemm_tflops / ceil_burst, "gemm_frac_of_sustained": gemm_tflops / ceil_sust,
+                                  "what": "back-to-back 256x256x64 pair MMAs on shared-memory-resident operands"}
+    clocks = sampler.stop(n_timed)
     ms_e2e, h2d, d2h = None, 0, 0
     if "e2e" in legs:
         # ---- e2e: host buffers, copies inside the timed region
