@@ -7,14 +7,17 @@
 // Shared memory (all 227 KB): six operand stages of 32 KB, a six-slot scale ring of 3 KB, 16 KB of epilogue staging.
 // TMEM: 256 accumulator columns + six scale slots of 24 columns.
 //
-// Roles per CTA (12 warps), all waits bounded as in gemm.cu:
+// Roles per CTA (12 warps in three warp groups), all waits bounded as in gemm.cu:
 //   warp 0       TMA producer: own A rows, own half of B (completion counted on the LEADER's barrier);
-//   warp 3       scale loader: own A-row scale tiles and the scale tiles of all 256 B rows, bulk copies into the ring;
-//                a ring slot is free as soon as the movers have carried it to TMEM, so the loads run two rings ahead;
-//   warps 1, 2   MMA issuers, leader CTA only, taking the K-steps in turn under a baton: four K = 64 pair-MMAs per
-//                step; ONE multicast tcgen05.commit per step frees operand stage and TMEM scale slot in BOTH CTAs;
-//   warps 8..11  scale movers: shared memory -> registers -> own TMEM lane quadrant (tcgen05.st); they arrive on the
-//                leader's full barrier of the stage, the same one the operand bytes complete, so the issuer waits once;
+//   warp 3       scale loader: own A-row scale tiles and the scale tiles of all 256 B rows, bulk copies into ring slot
+//                s of stage s (free again when the step's MMAs, and with them its scale copies, have completed);
+//   warps 1, 2   MMA issuers, leader CTA only, taking the K-steps in turn under a baton.  Per step: six tcgen05.cp
+//                carry the step's scale tiles from the ring into TMEM slot s of BOTH CTAs (the copy itself replicates
+//                them to the four lane quadrants and reads shared memory once; they are issued while the other
+//                thread still issues its MMAs), then four K = 64 pair-MMAs; ONE multicast tcgen05.commit per step
+//                frees operand stage, ring slot and TMEM scale slot in both CTAs;
+//   warp 8       forwards "this CTA's scale tiles of step i have landed" to the leader's full barrier of the stage,
+//                the same one the operand bytes complete, so the issuer waits once (warps 9..11 only fill the group);
 //   warps 4..7   epilogue of the CTA's own 128 x 256 half tile: accumulator -> registers (packed bf16) -> hand the
 //                accumulator back -> swizzled staging -> TMA stores (or reduce-adds when accumulating).
 // A-row scales are per CTA; every CTA needs the scales of all 256 B rows.
@@ -44,9 +47,9 @@ constexpr uint32_t kSmemP = kStagesP * kStageB + kSfSlotsP * kSfSlotB + kEpiB + 
 static_assert(kSmemP <= 232448, "over the 227 KB shared-memory limit");
 constexpr uint32_t kAccColP = 0, kSfColP = 256, kSfSlotColsP = 24;
 constexpr int kGroupMP = 8;                                 // rasterisation: 8 pair-tiles (2048 rows) share B tiles in L2
-// Register hand-over (setmaxnreg) between the three warp groups; an increase can only draw on what the CTA holds at
+// Register hand-over (setmaxnreg) between the three warp groups (kRegsFwdP: the forwarder's group); an increase can only draw on what the CTA holds at
 // launch (threads x registers per thread), which gemm_pair_init checks: an increase that cannot be met waits forever.
-constexpr int kRegsLightP = 56, kRegsMoverP = 64, kRegsEpiP = 232;
+constexpr int kRegsLightP = 56, kRegsFwdP = 64, kRegsEpiP = 232;
 constexpr int kThreadsP = 12 * 32;
 
 struct ParamsP {
@@ -79,12 +82,11 @@ gemm_mxf4_pair_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_c
     uint8_t* sf_ring = smem + kStagesP * kStageB;
     uint8_t* epi_ring = sf_ring + kSfSlotsP * kSfSlotB;
     uint64_t* bars = reinterpret_cast<uint64_t*>(epi_ring + kEpiB);
-    uint64_t* full_bar = bars;                              // [kStagesP] leader: operands of both CTAs landed AND their
-                                                            //            scales are in TMEM (1 expect_tx arrival + 8 movers)
+    uint64_t* full_bar = bars;                              // [kStagesP] leader: operands and scale tiles of both CTAs landed
+                                                            //            (1 expect_tx arrival + 1 forwarder per CTA)
     uint64_t* empty_bar = full_bar + kStagesP;              // [kStagesP] per CTA: stage and scale slot free (pair commit)
     uint64_t* sfl_full = empty_bar + kStagesP;              // [kSfSlotsP] per CTA: scale tiles landed in the ring slot
-    uint64_t* sfl_empty = sfl_full + kSfSlotsP;             // [kSfSlotsP] per CTA: the movers have read the ring slot (4 arrivals)
-    uint64_t* turn = sfl_empty + kSfSlotsP;                 // [2] leader: baton between the two MMA issuers
+    uint64_t* turn = sfl_full + kSfSlotsP;                 // [2] leader: baton between the two MMA issuers
     uint64_t* tmem_full = turn + 2;                         // per CTA: accumulator complete (pair commit)
     uint64_t* tmem_empty = tmem_full + 1;                   // leader: both CTAs drained their accumulators
     uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(tmem_empty + 1);
@@ -100,8 +102,8 @@ gemm_mxf4_pair_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_c
     const uint32_t total = my_tiles * (uint32_t)num_kt;
 
     if (threadIdx.x == 0) {
-        for (int s = 0; s < kStagesP; ++s) { mbar_init(&full_bar[s], 1 + 8); mbar_init(&empty_bar[s], 1); }
-        for (int s = 0; s < kSfSlotsP; ++s) { mbar_init(&sfl_full[s], 1); mbar_init(&sfl_empty[s], 4); }
+        for (int s = 0; s < kStagesP; ++s) { mbar_init(&full_bar[s], 1 + 2); mbar_init(&empty_bar[s], 1); }
+        for (int s = 0; s < kSfSlotsP; ++s) mbar_init(&sfl_full[s], 1);
         mbar_init(&turn[0], 1); mbar_init(&turn[1], 1);
         mbar_init(tmem_full, 1);
         mbar_init(tmem_empty, 8);
@@ -120,7 +122,7 @@ gemm_mxf4_pair_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_c
     cluster_sync_all();                                     // both CTAs' barriers exist before anyone signals across
     tc_fence_after_sync();
     const uint32_t tmem_base = *tmem_slot;
-    // Warp group 0 (producer, issuers, scale loader) and warp group 2 (scale movers) need few registers; the epilogue
+    // Warp group 0 (producer, issuers, scale loader) and warp group 2 (forwarder) need few registers; the epilogue
     // group takes them to hold half an accumulator row and four TMEM loads in flight.
     // Each warp group (four warps) sets its register limit once, at the head of its own branch: all four warps must
     // execute the same setmaxnreg, and the limit must dominate the code that relies on it.
@@ -171,14 +173,27 @@ gemm_mxf4_pair_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_c
             while (kt >= num_kt) { kt -= num_kt; ++tile_i; }
             bool ok = true;
             for (uint32_t it = me; it < total; it += 2, ++n) {
-                if (kt == 0) {
-                    if (!(ok = mbar_wait(tmem_empty, (tile_i & 1) ^ 1, abort_flag))) break;
-                }
                 if (!(ok = mbar_wait(&full_bar[s], ph, abort_flag))) break;
-                if (!(ok = mbar_wait_spin(&turn[me], (n & 1) ^ me ^ 1, abort_flag))) break;   // the step before mine is issued
                 tc_fence_after_sync();
                 const uint32_t a_lo = a_lo0 + s * (kStageB >> 4), b_lo = a_lo + (kAB >> 4);
                 const uint32_t sfa_t = tmem_base + kSfColP + s * kSfSlotColsP, sfb_t = sfa_t + 8;
+                {   // the step's scales: shared memory -> TMEM of both CTAs, replicated to the four lane quadrants by the copy;
+                    // issued while the other thread still issues its MMAs (a different TMEM slot), ordered before this
+                    // thread's MMAs by program order
+                    const uint32_t sf_s = smem_u32(sf_ring + s * kSfSlotB);
+#pragma unroll
+                    for (int c = 0; c < 2; ++c) {
+                        tc_cp_32x128b_warpx4_pair(sfa_t + 4 * c, make_smem_desc(sf_s + c * kSfTile, 0, 128, 0));
+#pragma unroll
+                        for (int j = 0; j < 2; ++j)
+                            tc_cp_32x128b_warpx4_pair(sfb_t + 8 * c + 4 * j, make_smem_desc(sf_s + kSfaB + (2 * j + c) * kSfTile, 0, 128, 0));
+                    }
+                }
+                if (kt == 0) {                                                   // the copies above did not need the accumulator
+                    if (!(ok = mbar_wait(tmem_empty, (tile_i & 1) ^ 1, abort_flag))) break;
+                    tc_fence_after_sync();
+                }
+                if (!(ok = mbar_wait_spin(&turn[me], (n & 1) ^ me ^ 1, abort_flag))) break;   // the step before mine is issued
                 const uint32_t hi2 = 2u << 30;
                 const bool last = kt == num_kt - 1;
                 auto D = [&](uint32_t lo) { return ((uint64_t)desc_hi << 32) | lo; };
@@ -212,8 +227,8 @@ gemm_mxf4_pair_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_c
                 const int n_row_tiles = min(2, (int)((p.N - (int64_t)nt * PN + 127) >> 7));
                 for (int kt = 0; kt < num_kt; ++kt, ++it) {
                     const int slot = it % kSfSlotsP;
-                    // the ring slot is free once the movers have carried its previous contents to TMEM
-                    if (!(ok = mbar_wait(&sfl_empty[slot], ((it / kSfSlotsP) & 1) ^ 1, abort_flag))) break;
+                    // the ring slot is free once the MMAs of the step that used it (and their scale copies) have completed
+                    if (!(ok = mbar_wait(&empty_bar[slot], ((it / kSfSlotsP) & 1) ^ 1, abort_flag))) break;
                     uint8_t* dst = sf_ring + slot * kSfSlotB;
                     const int nch = min(2, nkc - 2 * kt);
                     mbar_expect_tx(&sfl_full[slot], (uint32_t)nch * kSfTile * ((has_a ? 1u : 0u) + (uint32_t)n_row_tiles));
@@ -227,30 +242,17 @@ gemm_mxf4_pair_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_c
         }
     }
     } else if (warp >= 8) {
-        // ============================ warp group 2: scale movers
-        reg_dealloc<kRegsMoverP>();
-        // ------------------------------------------------------------------ scale movers (both CTAs, warps 6..9)
-        const int q = warp & 3;
-        const uint32_t lane_base = (uint32_t)(q * 32) << 16;
+        // ============================ warp group 2: scale forwarder (warp 8)
+        reg_dealloc<kRegsFwdP>();
+        // The scale copies run in both CTAs on the leader's instruction, so the leader has to know that the peer's tiles
+        // have landed too: one thread per CTA passes its ring's completions on to the leader's full barrier.
         bool ok = true;
-        for (uint32_t it = 0; it < total; ++it) {
-            const int slot = it % kSfSlotsP;
-            if (lane == 0) {
-                // scales landed in shared memory, and the MMAs that read this TMEM slot's previous scales are done
-                ok = mbar_wait(&sfl_full[slot], (it / kSfSlotsP) & 1, abort_flag) &&
-                     mbar_wait(&empty_bar[slot], ((it / kSfSlotsP) & 1) ^ 1, abort_flag);
+        if (warp == 8 && lane == 0) {
+            for (uint32_t it = 0; it < total; ++it) {
+                const int slot = it % kSfSlotsP;
+                if (!(ok = mbar_wait(&sfl_full[slot], (it / kSfSlotsP) & 1, abort_flag))) break;
+                mbar_arrive_cluster(&full_bar[slot], 0);
             }
-            ok = __shfl_sync(0xffffffffu, ok, 0);
-            if (!ok) break;
-            tc_fence_after_sync();
-            const uint4* sf = reinterpret_cast<const uint4*>(sf_ring + slot * kSfSlotB) + lane;          // 32 uint4 per tile
-            const uint32_t sfa_t = tmem_base + lane_base + kSfColP + slot * kSfSlotColsP, sfb_t = sfa_t + 8;
-            tmem_st_32x32b_x8(sfa_t, sf[0], sf[32]);
-            tmem_st_32x32b_x16(sfb_t, sf[64], sf[128], sf[96], sf[160]);
-            tmem_st_wait();
-            tc_fence_before_sync();
-            __syncwarp();
-            if (lane == 0) { mbar_arrive(&sfl_empty[slot]); mbar_arrive_cluster(&full_bar[slot], 0); }
         }
         if (!ok && lane == 0) *abort_flag = 1;
     } else {
@@ -422,7 +424,7 @@ cudaError_t gemm_pair_init() {
     cudaFuncAttributes fa;
     e = cudaFuncGetAttributes(&fa, gemm_mxf4_pair_kernel);
     if (e != cudaSuccess) return e;
-    if (fa.numRegs * kThreadsP < 128 * (kRegsLightP + kRegsMoverP + kRegsEpiP)) return cudaErrorLaunchOutOfResources;
+    if (fa.numRegs * kThreadsP < 128 * (kRegsLightP + kRegsFwdP + kRegsEpiP)) return cudaErrorLaunchOutOfResources;
     return cudaSuccess;
 }
 
