@@ -37,7 +37,7 @@ BF16_TO_FP4 = 4.0                    # nominal dense ratio 9 / 2.25 PFLOP/s
 QUANT_BYTES_PER_ELEM = 2.0 + 0.5 + 1.0 / 32.0   # bf16 in, E2M1 code + E8M0 scale out
 # DRAM bytes moved / algorithmic bytes of the GEMM, from one ncu capture (profiles/gemm_mxf4_pair_16384x4096x16384.md:
 # 477.8 MB measured against 312.6 MB of codes, scales and bf16 output); applied to the average launch of the step.
-GEMM_TRAFFIC_OVER_ALGORITHMIC = 1.49
+GEMM_TRAFFIC_OVER_ALGORITHMIC = 1.50
 ROUNDINGS = {"sr": 0, "rn": 1, "sr16": 2}      # the C ABI's and the oracle's rounding selectors
 
 
@@ -444,7 +444,7 @@ def run_gpu(args):
                          "kernel": "gemm_mxf4_pair_kernel", "bound": "tensor", "achieved": gemm_tflops, "peak": fp4_peak, "unit": "TFLOP/s",
                          "frac": gemm_tflops / fp4_peak,
                          "traffic": GEMM_TRAFFIC_OVER_ALGORITHMIC * gemm_bytes / gemm_n,
-                         "traffic_note": "bytes per average launch = algorithmic bytes x 1.49 (ratio from an ncu capture of the 16384x4096x16384 launch)",
+                         "traffic_note": "bytes per average launch = algorithmic bytes x 1.50 (ratio from an ncu capture of the 16384x4096x16384 launch)",
                          "peak_source": f"4 x {peaks['source']} sustained bf16 ({peaks['bf16_sustained']} TFLOP/s); no FP4 peak was measured"},
             "kernels": kernels,
             "variants": variants,
