@@ -78,6 +78,50 @@ __device__ __forceinline__ void sr_draws32(const PhiloxKeys& ks, uint32_t stream
     rw[4] = b.x; rw[5] = b.y; rw[6] = b.z; rw[7] = b.w;
 }
 
+// The SR draws of one operand view share seed and stream tag, and for operands below 2^36 elements the high counter
+// word is zero: the counter is (index, 0, tag, 1).  Everything in the first three rounds that does not depend on the
+// index is folded into five words per view (computed on the host with the key schedule): the rounds themselves, and so
+// the draws, are unchanged.
+struct PhiloxViewConsts {
+    uint32_t c1, d, e, f, qlo;
+};
+__host__ __device__ inline PhiloxViewConsts philox_view_consts(const PhiloxKeys& ks, uint32_t stream_tag) {
+    const unsigned long long p1 = 0xCD9E8D57ull * stream_tag;             // round 1: second product, counter word 2 = tag
+    const uint32_t a = (uint32_t)(p1 >> 32) ^ 0u ^ ks.k0[0], b = (uint32_t)p1;   // new words 0, 1 (counter word 1 = 0)
+    const unsigned long long q = 0xD2511F53ull * a;                       // round 2: first product
+    PhiloxViewConsts v;
+    v.c1 = 1u ^ ks.k1[0];                                                 // round 1, word 2: hi(M0 x0) ^ (domain 1) ^ key
+    v.d = b ^ ks.k0[1];                                                   // round 2, word 0: hi(M1 y2) ^ b ^ key
+    v.e = (uint32_t)(q >> 32) ^ ks.k1[1];                                 // round 2, word 2: y3 ^ hi(M0 a) ^ key
+    v.qlo = (uint32_t)q;                                                  // round 2, word 3
+    v.f = v.qlo ^ ks.k1[2];                                               // round 3, word 2: hi(M0 z0) ^ qlo ^ key
+    return v;
+}
+__device__ __forceinline__ uint4 philox4x32_10_view(uint32_t x0, const PhiloxViewConsts& v, const PhiloxKeys& ks) {
+    const uint32_t y2 = __umulhi(0xD2511F53u, x0) ^ v.c1, y3 = 0xD2511F53u * x0;                 // round 1
+    const uint32_t z0 = __umulhi(0xCD9E8D57u, y2) ^ v.d, z1 = 0xCD9E8D57u * y2, z2 = y3 ^ v.e;   // round 2
+    uint32_t c0 = __umulhi(0xCD9E8D57u, z2) ^ z1 ^ ks.k0[2], c1 = 0xCD9E8D57u * z2;              // round 3
+    uint32_t c2 = __umulhi(0xD2511F53u, z0) ^ v.f, c3 = 0xD2511F53u * z0;
+#pragma unroll
+    for (int i = 3; i < 10; ++i) {
+        const uint32_t hi0 = __umulhi(0xD2511F53u, c0), lo0 = 0xD2511F53u * c0;
+        const uint32_t hi1 = __umulhi(0xCD9E8D57u, c2), lo1 = 0xCD9E8D57u * c2;
+        c0 = hi1 ^ c1 ^ ks.k0[i];
+        c1 = lo1;
+        c2 = hi0 ^ c3 ^ ks.k1[i];
+        c3 = lo0;
+    }
+    return make_uint4(c0, c1, c2, c3);
+}
+// The 32 draws of elements [i0, i0 + 32), i0 a multiple of 32 below 2^36.
+__device__ __forceinline__ void sr_draws32_view(const PhiloxKeys& ks, const PhiloxViewConsts& v, uint64_t i0, uint32_t (&rw)[8]) {
+    const uint32_t lo = (uint32_t)(i0 >> 4);
+    const uint4 a = philox4x32_10_view(lo, v, ks);
+    const uint4 b = philox4x32_10_view(lo | 1u, v, ks);
+    rw[0] = a.x; rw[1] = a.y; rw[2] = a.z; rw[3] = a.w;
+    rw[4] = b.x; rw[5] = b.y; rw[6] = b.z; rw[7] = b.w;
+}
+
 // ---------------------------------------------------------------- Hadamard butterflies (Eq. 4)
 // In-place Sylvester transform over the 32 values of one thread (natural order, un-normalised).
 __device__ __forceinline__ void fwht32(float (&v)[32]) {

@@ -58,6 +58,7 @@ struct QView {                 // one operand view: output operand [R, K] read f
     uint32_t d_major, d_minor; // an epilogue group's stride through the tile list, split by minor_count
     int reduce_dim;            // 1: K runs along x columns (x tile is the K-major operand); 0: along x rows (MN-major)
     uint32_t stream_tag;
+    PhiloxViewConsts pv;       // index-independent part of the first three Philox rounds for this view's draws (operands < 2^36 elements)
     uint8_t* codes;
     uint8_t* scales;
     float* y_out;              // transform dump only
@@ -116,6 +117,14 @@ constexpr bool mode_draws(int mode) { return mode == kModeSR || mode == kModeSR1
 // template argument of quantize_block32_rw; the g = 256 kernel (kw = 2) rounds SR through the convert instruction (same codes, fewer registers)
 constexpr int mode_rounding(int mode, int kw) { return mode == kModeSR16 ? 2 : (mode == kModeSR && kw == 2) ? 3 : mode; }
 
+// The 32 draws of a block.  FOLD: with the view's precomputed constants (fewer instructions, five more live values: pays
+// where registers are not the limit, i.e. in the SR16 kernel; the integer SR path and the g = 256 kernel lose with it).
+template <bool FOLD>
+__device__ __forceinline__ void view_draws32(const PhiloxKeys& ks, uint32_t stream_tag, const PhiloxViewConsts* pv, uint64_t i0, uint32_t (&rw)[8]) {
+    if (FOLD) sr_draws32_view(ks, *pv, i0, rw);
+    else sr_draws32(ks, stream_tag, i0, rw);
+}
+
 // KW = 128-wide k-tiles per entry of the tile list: 1, or 2 for g = 256 (a tile then spans one 256-chunk).
 template <int MODE, int KW>
 __global__ void __launch_bounds__(kThreadsQ, 1)
@@ -133,6 +142,7 @@ quantize_tc_kernel(const __grid_constant__ QMaps maps, const __grid_constant__ Q
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const uint32_t num_tiles = p.n_tiles;
+    constexpr bool kFold = MODE == kModeSR16 && KW == 1;
 
     if (threadIdx.x == 0) {
         for (int s = 0; s < kStagesQ; ++s) { mbar_init(&full_bar[s], 1); mbar_init(&empty_bar[s], 1); }
@@ -263,7 +273,7 @@ quantize_tc_kernel(const __grid_constant__ QMaps maps, const __grid_constant__ Q
         uint32_t t = blockIdx.x + it * gridDim.x;
         TilePos pos = locate_tile(p, t < num_tiles ? t : 0u);
         uint32_t rw[8];
-        if (mode_draws(MODE)) sr_draws32(p.keys, p.view[pos.v].stream_tag, first_elem(pos), rw);
+        if (mode_draws(MODE)) view_draws32<kFold>(p.keys, p.view[pos.v].stream_tag, &p.view[pos.v].pv, first_elem(pos), rw);
         if (KW == 2) {
             // g = 256: a tile is one 256-chunk of 128 rows; its two k-tiles went through T_0 and T_1 into the accumulator
             // pair (b0, b0 + 1): u = A_lo T_0, v = A_hi T_1.  The transformed values are y[0..127] = u + v and
@@ -275,7 +285,7 @@ quantize_tc_kernel(const __grid_constant__ QMaps maps, const __grid_constant__ Q
             it = (uint32_t)pr;
             t = blockIdx.x + it * gridDim.x;
             pos = locate_tile(p, t < num_tiles ? t : 0u);
-            if (mode_draws(MODE)) sr_draws32(p.keys, p.view[pos.v].stream_tag, first_elem(pos) + 128u * hh, rw);
+            if (mode_draws(MODE)) view_draws32<kFold>(p.keys, p.view[pos.v].stream_tag, &p.view[pos.v].pv, first_elem(pos) + 128u * hh, rw);
             for (; t < num_tiles; t += stride2, it += 2) {
                 const int b0 = 2 * pr;
                 const QView& vw = p.view[pos.v];
@@ -290,9 +300,11 @@ quantize_tc_kernel(const __grid_constant__ QMaps maps, const __grid_constant__ Q
                 float* y_dst = MODE == kModeDump ? vw.y_out + row * K + k0 : nullptr;
                 const uint64_t i_cur = first_elem(pos) + 128u * hh;
                 const uint32_t tag_cur = vw.stream_tag;
+                const PhiloxViewConsts* pv_cur = &vw.pv;
                 pos = t + stride2 < num_tiles ? advance_tile(p, pos, t + stride2) : locate_tile(p, 0u);
                 const uint64_t i_next = first_elem(pos) + 128u * hh;
                 const uint32_t tag_next = p.view[pos.v].stream_tag;
+            const PhiloxViewConsts* pv_next = &p.view[pos.v].pv;
                 const uint32_t ph = (it >> 1) & 1;                               // this pair's (it / 2)-th use
                 ok = mbar_wait(&acc_full[b0], ph, abort_flag) && mbar_wait(&acc_full[b0 + 1], ph, abort_flag);
                 ok = __all_sync(0xffffffffu, ok);
@@ -320,8 +332,8 @@ quantize_tc_kernel(const __grid_constant__ QMaps maps, const __grid_constant__ Q
                         if (lane == 0) { mbar_arrive(&acc_empty[b0]); mbar_arrive(&acc_empty[b0 + 1]); }
                     }
                     if (mode_draws(MODE)) {
-                        if (j < 3) sr_draws32(p.keys, tag_cur, i_cur + 32 * (j + 1), nx);
-                        else sr_draws32(p.keys, tag_next, i_next, nx);
+                        if (j < 3) view_draws32<kFold>(p.keys, tag_cur, pv_cur, i_cur + 32 * (j + 1), nx);
+                        else view_draws32<kFold>(p.keys, tag_next, pv_next, i_next, nx);
                     }
                     if (MODE == kModeDump) {
                         if (live) {
@@ -356,10 +368,12 @@ quantize_tc_kernel(const __grid_constant__ QMaps maps, const __grid_constant__ Q
             float* y_dst = MODE == kModeDump ? vw.y_out + row * K + k0 : nullptr;
             const uint64_t i_cur = first_elem(pos);
             const uint32_t tag_cur = vw.stream_tag;
+            const PhiloxViewConsts* pv_cur = &vw.pv;
             // position of the next tile of this group (past the end: computed but not used)
             pos = t + stride < num_tiles ? advance_tile(p, pos, t + stride) : locate_tile(p, 0u);
             const uint64_t i_next = first_elem(pos);
             const uint32_t tag_next = p.view[pos.v].stream_tag;
+            const PhiloxViewConsts* pv_next = &p.view[pos.v].pv;
             ok = mbar_wait(&acc_full[b], (it / kAccBufs) & 1, abort_flag);
             ok = __all_sync(0xffffffffu, ok);
             if (!ok) break;
@@ -378,8 +392,8 @@ quantize_tc_kernel(const __grid_constant__ QMaps maps, const __grid_constant__ Q
                     if (lane == 0) mbar_arrive(&acc_empty[b]);
                 }
                 if (mode_draws(MODE)) {
-                    if (j < 3) sr_draws32(p.keys, tag_cur, i_cur + 32 * (j + 1), nx);
-                    else sr_draws32(p.keys, tag_next, i_next, nx);
+                    if (j < 3) view_draws32<kFold>(p.keys, tag_cur, pv_cur, i_cur + 32 * (j + 1), nx);
+                    else view_draws32<kFold>(p.keys, tag_next, pv_next, i_next, nx);
                 }
 #pragma unroll
                 for (int i = 0; i < 32; ++i) y[i] = __uint_as_float(raw[i]);
@@ -427,7 +441,9 @@ bool quant_tc_eligible(const QuantArgs& a) {
     const int64_t K = a.reduce_dim == 1 ? a.cols : a.rows;
     const int64_t R = a.reduce_dim == 1 ? a.rows : a.cols;
     const int64_t tiles = ((R + kTile - 1) / kTile) * (K / kTile);          // tile indices are 32-bit in the kernel
-    return (a.g == 32 || a.g == 64 || a.g == 128 || a.g == 256) && K % kTile == 0 && tiles < (int64_t(1) << 28) && a.has_tmap;
+    // the element index that keys the SR draws stays below 2^36 (the kernel folds a zero high counter word into its constants)
+    return (a.g == 32 || a.g == 64 || a.g == 128 || a.g == 256) && K % kTile == 0 && tiles < (int64_t(1) << 28) && a.has_tmap &&
+           R * K < (int64_t(1) << 36);
 }
 
 cudaError_t fetch_quant_tc_status(unsigned int* word) { return device_status_fetch(word); }
@@ -481,6 +497,7 @@ cudaError_t launch_quantize_tc_group(const QuantArgs* a, int n, bool dump_y, cud
             k0 += 0x9E3779B9u; k1 += 0xBB67AE85u;
         }
     }
+    for (int v = 0; v < kQuantMaxViews; ++v) p.view[v].pv = philox_view_consts(p.keys, p.view[v].stream_tag);
     int dev = 0, sms = 0;
     cudaError_t e = cudaGetDevice(&dev);
     if (e != cudaSuccess) return e;
