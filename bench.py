@@ -293,6 +293,23 @@ def run_gpu(args):
         for kind, name, a, b, work in records:
             d = agg.setdefault(kind, [0.0, 0.0, 0])
             d[0] += a.elapsed_time(b) * 1e-3; d[1] += work; d[2] += 1
+        # the three lines per layer: quantiser alone (GB/s, of HBM peak), GEMMs alone on the quantised operands
+        # (TFLOP/s, of the FP4 peaks), and the layer end to end = 4bmn / (its three launches)
+        per_layer = {}
+        for kind, name, a, b, work in records:
+            d = per_layer.setdefault(name, {"quant_s": 0.0, "quant_bytes": 0.0, "gemm_s": 0.0, "flops": 0.0})
+            t = a.elapsed_time(b) * 1e-3
+            if kind == "quant":
+                d["quant_s"] += t; d["quant_bytes"] += work
+            else:
+                d["gemm_s"] += t; d["flops"] += work
+        for name, d in per_layer.items():
+            q_gbs, g_tf = d["quant_bytes"] / d["quant_s"] / 1e9, d["flops"] / d["gemm_s"] / 1e12
+            per_layer[name] = {"quant_GB/s": q_gbs, "quant_frac_of_hbm_peak": q_gbs / peaks["hbm_gbs"],
+                               "gemm_TFLOP/s": g_tf, "gemm_frac_of_4x_bf16_sustained": g_tf / fp4_peak,
+                               "gemm_frac_of_nominal_9pf": g_tf / NOMINAL_FP4_TFLOPS,
+                               "layer_TFLOP/s": d["flops"] / (d["quant_s"] + d["gemm_s"]) / 1e12,
+                               "ms": (d["quant_s"] + d["gemm_s"]) / k_roof * 1e3}
         gemm_t, gemm_fl, gemm_n = agg["gemm"]
         gemm_bytes = k_roof * sum((l.b * l.m + l.n * l.m) * 0.53125 + l.b * l.n * 2 + (l.m * l.b + l.n * l.b) * 0.53125 + l.m * l.n * 2
                                   for l in layers)
@@ -306,6 +323,7 @@ def run_gpu(args):
                            "frac_of_4x_bf16_sustained": gemm_tflops / fp4_peak,
                            "frac_of_4x_bf16_burst": gemm_tflops / (BF16_TO_FP4 * peaks["bf16_burst"]),
                            "frac_of_nominal_9pf": gemm_tflops / NOMINAL_FP4_TFLOPS}
+        kernels["per_layer"] = per_layer
         calls_ms = sum(v[0] for v in agg.values()) / k_roof * 1e3
     variants = {}
     if "roofline" in legs:
