@@ -212,6 +212,25 @@ ORC_API int orc_rht(const uint16_t *x, int64_t R, int64_t K, int64_t stride_r, i
 /* ------------------------------------------------------------------------- */
 
 /* 1 sign, 2 exponent (bias 1), 1 mantissa bit.  Magnitudes by code 0..7. */
+/* Section 3.2, last paragraph: the blockwise construction works with ANY orthogonal g x g matrix in place of
+ * diag(S) H_g / sqrt(g).  Every contiguous g-chunk v of a row becomes y_j = sum_i v_i T[i][j], T given as bf16
+ * (raw 16-bit patterns, row-major g x g): explicit product in fp64, rounded once to fp32. */
+ORC_API int orc_transform(const uint16_t *x, int64_t R, int64_t K, int64_t stride_r, int64_t stride_k,
+                          int g, const uint16_t *T, float *y /* [R, K] row-major */)
+{
+    if (g < 1 || K % g != 0) return -1;
+#pragma omp parallel for schedule(static)
+    for (int64_t r = 0; r < R; ++r)
+        for (int64_t c = 0; c < K / g; ++c)
+            for (int j = 0; j < g; ++j) {
+                double acc = 0.0;
+                for (int i = 0; i < g; ++i)
+                    acc += bf16_to_double(x[r * stride_r + (c * g + i) * stride_k]) * bf16_to_double(T[i * g + j]);
+                y[r * K + c * g + j] = (float)acc;
+            }
+    return 0;
+}
+
 static const double E2M1_GRID[8] = { 0.0, 0.5, 1.0, 1.5, 2.0, 3.0, 4.0, 6.0 };
 
 ORC_API double orc_e2m1_value(uint32_t code)

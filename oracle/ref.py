@@ -30,6 +30,8 @@ _lib.orc_hadamard.argtypes = [C.c_int, _i8p]
 _lib.orc_hadamard.restype = C.c_int
 _lib.orc_rht.argtypes = [C.c_void_p, _i64, _i64, _i64, _i64, C.c_int, _u64, _f32p]
 _lib.orc_rht.restype = C.c_int
+_lib.orc_transform.argtypes = [C.c_void_p, _i64, _i64, _i64, _i64, C.c_int, C.c_void_p, _f32p]
+_lib.orc_transform.restype = C.c_int
 _lib.orc_e2m1_value.argtypes = [C.c_uint32]
 _lib.orc_e2m1_value.restype = C.c_double
 _lib.orc_e8m0_from_amax.argtypes = [C.c_float]
@@ -135,6 +137,16 @@ def rht(x: np.ndarray, g: int, seed: int, transpose: bool = False) -> np.ndarray
     ptr, R, K, sr, sk = _view(x, transpose)
     y = np.empty((R, K), np.float32)
     if _lib.orc_rht(ptr, R, K, sr, sk, g, seed, y) != 0:
+        raise ValueError("bad g / shape")
+    return y
+
+
+def transform(x: np.ndarray, T: np.ndarray, transpose: bool = False) -> np.ndarray:
+    """Blockwise transform with a given g x g matrix T (bf16 bits): every g-chunk v of the reduce dim becomes v T."""
+    ptr, R, K, sr, sk = _view(x, transpose)
+    assert T.dtype == np.uint16 and T.ndim == 2 and T.shape[0] == T.shape[1] and T.flags.c_contiguous
+    y = np.empty((R, K), np.float32)
+    if _lib.orc_transform(ptr, R, K, sr, sk, T.shape[0], T.ctypes.data, y) != 0:
         raise ValueError("bad g / shape")
     return y
 

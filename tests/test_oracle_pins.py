@@ -293,6 +293,35 @@ def test_sr_monte_carlo_through_philox(ref):
     assert np.all(np.abs(acc / T - 0.75 * y) <= 5 * sigma + X / 512)
 
 
+def test_transform_with_a_given_matrix(ref):
+    """Section 3.2: any orthogonal matrix may stand in for the RHT.  With T = diag(S) H_g / sqrt(g) (exact in bf16 for
+    g = 64) the given-matrix transform is the RHT; with the identity it is the input; with a random orthogonal Q (QR of
+    a Gaussian matrix, fp64) norms and products are preserved; bf16 rounding of Q costs about 2^-9."""
+    rng = np.random.default_rng(17)
+    x = wl.grad_like(rng, (64, 256), 1.0)
+    seed, g = 77, 64
+    S = ref.sign_vector(seed, g).astype(np.float64)
+    T = (S[:, None] * ref.hadamard(g).astype(np.float64)) / 8.0
+    Tb = wl.to_bf16_bits(T.astype(np.float32))
+    assert np.array_equal(wl.bf16_bits_to_f64(Tb), T)                      # +-1/8: exact
+    for tr in (False, True):
+        assert np.array_equal(ref.transform(x, Tb, transpose=tr), ref.rht(x, g, seed, transpose=tr))
+    eye = wl.to_bf16_bits(np.eye(32, dtype=np.float32))
+    assert np.array_equal(ref.transform(x, eye), wl.bf16_bits_to_f64(x).astype(np.float32))
+    Q, _ = np.linalg.qr(rng.standard_normal((32, 32)))
+    Qb = wl.to_bf16_bits(Q.astype(np.float32))
+    y = ref.transform(x, Qb).astype(np.float64)
+    xv = wl.bf16_bits_to_f64(x)
+    want = (xv.reshape(64, 8, 32) @ wl.bf16_bits_to_f64(Qb)).reshape(64, 256)       # numpy's own product with the same bf16 matrix
+    assert np.abs(y - want).max() <= 2.0 ** -23 * np.abs(want).max()
+    nx, ny = np.linalg.norm(xv.reshape(64, 8, 32), axis=2), np.linalg.norm(y.reshape(64, 8, 32), axis=2)
+    assert np.abs(ny / nx - 1).max() < 2.0 ** -6                           # orthogonal up to the bf16 rounding of Q
+    b = wl.weight_like(rng, (16, 256))
+    yb = ref.transform(b, Qb).astype(np.float64)
+    exact = xv @ wl.bf16_bits_to_f64(b).T
+    assert np.linalg.norm(y @ yb.T - exact) / np.linalg.norm(exact) < 2.0 ** -6
+
+
 # --------------------------------------------------------------------------- second SR reading (16-bit dither)
 
 def _rev(v, bits):
