@@ -98,6 +98,21 @@ MXFP4_API mxfp4_status mxfp4_rht(const void* x, int64_t rows, int64_t cols, int6
                        int g, uint64_t seed, float* y, void* cuda_stream);
 
 /*
+ * The same quantiser with a transform matrix given by the caller (Section 3.2: the blockwise construction works with
+ * any random orthogonal matrix, the RHT is one choice): every contiguous g-chunk v of the reduction dimension becomes
+ * v T before quantisation.
+ *   T      bf16 [g, g] row-major, DEVICE pointer, 16-byte aligned, g in {32, 64, 128}; applied as given (no 1/sqrt(g)).
+ *          The product of two operands is preserved only if both use the same T and T is orthogonal: the caller's duty.
+ *   y      NULL, or fp32 [R, K] out (16-byte aligned): then only the transform runs and codes / scales may be NULL.
+ *   seed, stream_tag: the SR draws only (there is no sign vector here).  K % 128 == 0 (tensor-core path only),
+ *   else MXFP4_ERR_SHAPE.  Everything else as mxfp4_rht_sr_quantize.
+ */
+MXFP4_API mxfp4_status mxfp4_transform_quantize(const void* x, int64_t rows, int64_t cols, int64_t ld, int reduce_dim,
+                                                int g, const void* T, int rounding, uint64_t seed, uint32_t stream_tag,
+                                                uint8_t* codes, uint8_t* scales, int sf_layout, float* y,
+                                                void* cuda_stream);
+
+/*
  * Block-scaled FP4 GEMM (MXFP4_GEMM of Algorithm 3 lines 7-8, with the 16/9 of lines 10-11 as alpha):
  *     C[M, N] = alpha * sum_k deq(A)[i, k] * deq(B)[j, k],   deq = E2M1 value * 2^(scale byte - 127)
  *   A_codes [M, K/2], B_codes [N, K/2] packed as above; A_scales / B_scales in the NATIVE layout

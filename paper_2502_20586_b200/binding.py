@@ -23,6 +23,8 @@ OUT_BF16, OUT_FP32 = 0, 1
 _vp, _i64, _u64, _u32, _int, _sz = C.c_void_p, C.c_int64, C.c_uint64, C.c_uint32, C.c_int, C.c_size_t
 _lib.mxfp4_rht_sr_quantize.argtypes = [_vp, _i64, _i64, _i64, _int, _int, _int, _u64, _u32, _vp, _vp, _int, _vp]
 _lib.mxfp4_rht_sr_quantize.restype = _int
+_lib.mxfp4_transform_quantize.argtypes = [_vp, _i64, _i64, _i64, _int, _int, _vp, _int, _u64, _u32, _vp, _vp, _int, _vp, _vp]
+_lib.mxfp4_transform_quantize.restype = _int
 _lib.mxfp4_rht.argtypes = [_vp, _i64, _i64, _i64, _int, _int, _u64, _vp, _vp]
 _lib.mxfp4_rht.restype = _int
 _lib.mxfp4_gemm.argtypes = [_vp, _vp, _vp, _vp, _i64, _i64, _i64, _int, C.c_float, _vp, _i64, _int, _vp]
@@ -57,7 +59,7 @@ _lib.mxfp4_status_string.restype = C.c_char_p
 EXPORTS = ["mxfp4_rht_sr_quantize", "mxfp4_rht", "mxfp4_gemm", "mxfp4_linear_backward_workspace",
            "mxfp4_linear_backward", "mxfp4_linear_backward_static", "mxfp4_scale_bytes", "mxfp4_device_status", "mxfp4_status_string",
            "mxfp4_fp4_ceiling", "mxfp4_linear_backward_ex_workspace", "mxfp4_linear_backward_ex", "mxfp4_gemm_fused",
-           "mxfp4_linear_backward_fused", "mxfp4_operand_layout", "mxfp4_quantize_operands"]
+           "mxfp4_linear_backward_fused", "mxfp4_operand_layout", "mxfp4_quantize_operands", "mxfp4_transform_quantize"]
 
 
 class MxFp4Error(RuntimeError):
@@ -112,6 +114,26 @@ def mxfp4_rht(x: torch.Tensor, reduce_dim: int, g: int, seed: int, y=None):
         y = torch.empty((R, K), dtype=torch.float32, device=x.device)
     _check(_lib.mxfp4_rht(_ptr(x), rows, cols, x.stride(0), reduce_dim, g, seed, _ptr(y), _stream()))
     return y
+
+
+def mxfp4_transform_quantize(x, reduce_dim: int, T, seed: int, stream_tag: int = 0, rounding: int = ROUND_SR,
+                             sf_layout: int = SF_NATIVE, dump: bool = False):
+    """Quantiser with a caller-given transform matrix T (bf16 [g, g]): (codes, scales), or the fp32 transform if dump."""
+    assert x.is_cuda and x.dtype == torch.bfloat16 and x.dim() == 2 and x.stride(1) == 1
+    assert T.is_cuda and T.dtype == torch.bfloat16 and T.dim() == 2 and T.shape[0] == T.shape[1] and T.is_contiguous()
+    rows, cols = x.shape
+    R, K = (rows, cols) if reduce_dim == 1 else (cols, rows)
+    g = T.shape[0]
+    if dump:
+        y = torch.empty((R, K), dtype=torch.float32, device=x.device)
+        _check(_lib.mxfp4_transform_quantize(_ptr(x), rows, cols, x.stride(0), reduce_dim, g, _ptr(T), rounding, seed, stream_tag,
+                                             0, 0, sf_layout, _ptr(y), _stream()))
+        return y
+    codes = torch.empty((R, K // 2), dtype=torch.uint8, device=x.device)
+    scales = torch.empty(mxfp4_scale_bytes(R, K, sf_layout), dtype=torch.uint8, device=x.device)
+    _check(_lib.mxfp4_transform_quantize(_ptr(x), rows, cols, x.stride(0), reduce_dim, g, _ptr(T), rounding, seed, stream_tag,
+                                         _ptr(codes), _ptr(scales), sf_layout, 0, _stream()))
+    return codes, scales
 
 
 def mxfp4_gemm(A_codes, A_scales, B_codes, B_scales, alpha: float = 1.0, out_dtype: int = OUT_BF16, C_out=None):

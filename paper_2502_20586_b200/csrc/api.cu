@@ -263,6 +263,24 @@ mxfp4_status mxfp4_rht(const void* x, int64_t rows, int64_t cols, int64_t ld, in
     return mx::launch_rht_dump(a, static_cast<cudaStream_t>(cuda_stream)) == cudaSuccess ? MXFP4_OK : MXFP4_ERR_CUDA;
 }
 
+mxfp4_status mxfp4_transform_quantize(const void* x, int64_t rows, int64_t cols, int64_t ld, int reduce_dim, int g, const void* T,
+                                      int rounding, uint64_t seed, uint32_t stream_tag, uint8_t* codes, uint8_t* scales,
+                                      int sf_layout, float* y, void* cuda_stream) {
+    if (T == nullptr || ((codes == nullptr || scales == nullptr) && y == nullptr)) return MXFP4_ERR_NULL;
+    mxfp4_status st = check_quant(x, rows, cols, ld, reduce_dim, g);
+    if (st != MXFP4_OK) return st;
+    if (g != 32 && g != 64 && g != 128) return MXFP4_ERR_BAD_G;
+    if (rounding != MXFP4_ROUND_SR && rounding != MXFP4_ROUND_RN && rounding != MXFP4_ROUND_SR16) return MXFP4_ERR_MODE;
+    if (sf_layout != MXFP4_SF_LINEAR && sf_layout != MXFP4_SF_NATIVE) return MXFP4_ERR_MODE;
+    if (!aligned16(T) || (codes && !aligned16(codes)) || (y && !aligned16(y))) return MXFP4_ERR_ALIGN;
+    if ((st = runtime_init()) != MXFP4_OK) return st;
+    QuantArgs a{x, rows, cols, ld, reduce_dim, g, rounding, seed, stream_tag, codes, scales, sf_layout == MXFP4_SF_NATIVE, y};
+    a.custom_t = T;
+    attach_input_map(a);
+    if (!mx::quant_tc_eligible(a)) return MXFP4_ERR_SHAPE;            // the given-matrix transform runs on the tensor-core path only
+    return mx::launch_quantize_tc(a, y != nullptr, static_cast<cudaStream_t>(cuda_stream)) == cudaSuccess ? MXFP4_OK : MXFP4_ERR_CUDA;
+}
+
 mxfp4_status mxfp4_gemm(const uint8_t* A_codes, const uint8_t* A_scales, const uint8_t* B_codes, const uint8_t* B_scales, int64_t M,
                         int64_t N, int64_t K, int sf_layout, float alpha, void* C, int64_t ldc, int out_dtype, void* cuda_stream) {
     if (!A_codes || !A_scales || !B_codes || !B_scales || !C) return MXFP4_ERR_NULL;

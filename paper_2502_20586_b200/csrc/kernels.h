@@ -20,6 +20,7 @@ struct QuantArgs {
     float* y_out;         // only for the transform dump
     CUtensorMap tmap_x;   // x as [rows, cols] bf16, box 64 cols x 128 rows, 128-byte swizzle (tensor-core path)
     bool has_tmap;
+    const void* custom_t = nullptr;   // bf16 [g, g] row-major: transform matrix given by the caller instead of diag(S) H_g / sqrt(g) (tensor-core path, g <= 128)
 };
 
 // Tensor-core transform path (quantize_tc.cu): g in {32, 64, 128} and reduce length a multiple of 128.

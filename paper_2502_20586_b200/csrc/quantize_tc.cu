@@ -69,6 +69,7 @@ struct QParams {
     int n_views;
     uint32_t n_tiles;          // over all views
     int g, sf_native;
+    const uint16_t* custom_t;  // bf16 [g, g] row-major transform matrix given by the caller, or null (then diag(S) H_g / sqrt(g))
     uint64_t seed;
     PipeConsts pipe;           // see quant_math.cuh: constants kept opaque to the compiler
     PhiloxKeys keys;           // the ten Philox round keys of `seed` (key schedule only; the rounds run on the device)
@@ -156,6 +157,7 @@ quantize_tc_kernel(const __grid_constant__ QMaps maps, const __grid_constant__ Q
         tmem_relinquish();
     }
     {
+        if (KW == 1 && p.custom_t != nullptr) pdl_wait();                // the matrix may come from the kernel before this one
         // Transform operand, written in the 128-byte-swizzled K-major layout the MMA descriptor expects:
         // entry (n, k) at box (k / 64), row n (128 B pitch), 16-byte chunk ((k % 64) / 8) ^ (n % 8).
 #pragma unroll
@@ -168,8 +170,17 @@ quantize_tc_kernel(const __grid_constant__ QMaps maps, const __grid_constant__ Q
 #pragma unroll
                 for (int j = 0; j < 4; ++j) {
                     const int k0 = c * 8 + 2 * j;
-                    w[j] = KW == 2 ? (transform_entry_256(n, k0, sign) | (transform_entry_256(n, k0 + 1, sign) << 16))
-                                   : (transform_entry(n, k0, p.g, sign) | (transform_entry(n, k0 + 1, p.g, sign) << 16));
+                    if (KW == 1 && p.custom_t != nullptr) {
+                        // entry (n, k) of the operand = T[k % g][n % g] inside a g-chunk, 0 across chunks (Section 3.2: any orthogonal matrix)
+                        const int gm = p.g - 1;
+                        const bool same = ((n ^ k0) & ~gm) == 0;              // k0 and k0 + 1 lie in the same chunk (g is even)
+                        const uint32_t lo = same ? p.custom_t[(k0 & gm) * p.g + (n & gm)] : 0u;
+                        const uint32_t hi = same ? p.custom_t[((k0 + 1) & gm) * p.g + (n & gm)] : 0u;
+                        w[j] = lo | (hi << 16);
+                    } else {
+                        w[j] = KW == 2 ? (transform_entry_256(n, k0, sign) | (transform_entry_256(n, k0 + 1, sign) << 16))
+                                       : (transform_entry(n, k0, p.g, sign) | (transform_entry(n, k0 + 1, p.g, sign) << 16));
+                    }
                 }
                 const uint32_t off = (uint32_t)(c >> 3) * kBoxBytes + (uint32_t)n * 128u + (uint32_t)(((c & 7) ^ (n & 7)) << 4);
                 *reinterpret_cast<uint4*>(smem_t + h * kTBytes + off) = make_uint4(w[0], w[1], w[2], w[3]);
@@ -260,7 +271,7 @@ quantize_tc_kernel(const __grid_constant__ QMaps maps, const __grid_constant__ Q
         const int e = warp - 4;
         const int q = warp & 3;                      // TMEM lane quadrant this warp may read
         const int grp = e >> 2;
-        const float cg = p.g == 32 ? 0.17677669529663687f : p.g == 128 ? 0.08838834764831845f : 1.0f;
+        const float cg = p.custom_t != nullptr ? 1.0f : p.g == 32 ? 0.17677669529663687f : p.g == 128 ? 0.08838834764831845f : 1.0f;
         const uint32_t stride = (uint32_t)kEpiGroups * gridDim.x;
         const uint32_t lane_row = (uint32_t)(q * 32 + lane);
         bool ok = true;
@@ -489,6 +500,8 @@ cudaError_t launch_quantize_tc_group(const QuantArgs* a, int n, bool dump_y, cud
     p.n_views = n;
     p.n_tiles = tiles;
     p.g = a[0].g; p.sf_native = a[0].sf_native; p.seed = a[0].seed;
+    p.custom_t = static_cast<const uint16_t*>(a[0].custom_t);
+    if (p.custom_t != nullptr && p.g == 256) return cudaErrorInvalidValue;
     p.pipe = make_pipe_consts();
     {   // Philox key schedule: key_i = key_0 + i * (0x9E3779B9, 0xBB67AE85)
         uint32_t k0 = (uint32_t)p.seed, k1 = (uint32_t)(p.seed >> 32);

@@ -120,6 +120,16 @@ def test_argument_validation_needs_no_device(lib):
     assert list(off) == sorted(off) and off[0] == 0 and all(o % 1024 == 0 for o in off)
     assert off[7] + lib.mxfp4_scale_bytes(512, 256) <= raw.mxfp4_linear_backward_workspace(256, 512, 512)
     assert off[1] - off[0] >= 256 * 512 // 2 and off[2] - off[1] >= lib.mxfp4_scale_bytes(256, 512)
+    # quantiser with a given transform matrix
+    tq = raw.mxfp4_transform_quantize
+    #      x  rows cols ld  rd g   T  rnd seed tag codes scales layout y stream
+    assert tq(P, 128, 256, 256, 1, 64, 0, 0, 0, 1, P, P, 1, 0, 0) == 1            # T NULL
+    assert tq(P, 128, 256, 256, 1, 64, P, 0, 0, 1, 0, P, 1, 0, 0) == 1            # neither codes nor y
+    assert tq(P, 128, 256, 256, 1, 256, P, 0, 0, 1, P, P, 1, 0, 0) == 4           # g = 256 not taken
+    assert tq(P, 128, 256, 256, 1, 0, P, 0, 0, 1, P, P, 1, 0, 0) == 4
+    assert tq(P, 128, 256, 256, 1, 64, P + 2, 0, 0, 1, P, P, 1, 0, 0) == 3        # T alignment
+    assert tq(P, 128, 256, 256, 1, 64, P, 4, 0, 1, P, P, 1, 0, 0) == 5            # rounding
+    assert tq(P, 128, 250, 256, 1, 64, P, 0, 0, 1, P, P, 1, 0, 0) == 2            # K % 32
     # measurement aid
     assert raw.mxfp4_fp4_ceiling(0, C.byref(C.c_int64(0)), 0) == 2
     assert raw.mxfp4_fp4_ceiling(64, None, 0) == 2

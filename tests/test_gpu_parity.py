@@ -371,3 +371,35 @@ def test_split_form_equals_the_one_call_form(gpu):
             assert torch.equal(c, q[i][0])
             assert np.array_equal(hp.sf_native_to_linear(s.cpu().numpy(), R, K), hp.sf_native_to_linear(q[i][1].cpu().numpy(), R, K))
     assert gpu.mxfp4_device_status() == 0
+
+
+@pytest.mark.parametrize("reduce_dim,shape", [(1, (200, 1280)), (0, (640, 136))])
+def test_quantiser_with_a_given_transform_matrix(gpu, ref, reduce_dim, shape):
+    """Section 3.2: any orthogonal matrix may replace the RHT.  (a) Given T = diag(S) H_64 / 8 (exact in bf16) the call
+    reproduces the RHT quantiser bit for bit; (b) with a random orthogonal matrix (bf16-rounded) the transform matches
+    the oracle's explicit product to 1e-5 per chunk and the codes are the oracle's on the GPU's own fp32 values."""
+    import torch
+    x = _inputs("grad", shape, 23)
+    seed = 1234
+    S = ref.sign_vector(seed, 64).astype(np.float64)
+    T = wl.to_bf16_bits(((S[:, None] * ref.hadamard(64)) / 8.0).astype(np.float32))
+    for rounding in (0, 2):
+        c, s = gpu.mxfp4_transform_quantize(_dev(x), reduce_dim, _dev(T), seed, 3, rounding, gpu.SF_LINEAR)
+        c0, s0 = gpu.mxfp4_rht_sr_quantize(_dev(x), reduce_dim, 64, seed, 3, rounding, gpu.SF_LINEAR)
+        assert torch.equal(c, c0) and torch.equal(s, s0)
+    rng = np.random.default_rng(29)
+    for g in (32, 128):
+        Q, _ = np.linalg.qr(rng.standard_normal((g, g)))
+        Qb = wl.to_bf16_bits(Q.astype(np.float32))
+        y_gpu = gpu.mxfp4_transform_quantize(_dev(x), reduce_dim, _dev(Qb), seed, 5, dump=True).cpu().numpy()
+        y_ref = ref.transform(x, Qb, transpose=(reduce_dim == 0)).astype(np.float64)
+        R, K = y_ref.shape
+        d = (y_gpu.astype(np.float64) - y_ref).reshape(R, K // g, g)
+        rel = np.linalg.norm(d, axis=2) / np.maximum(np.linalg.norm(y_ref.reshape(R, K // g, g), axis=2), 1e-300)
+        assert rel.max() <= 1e-5
+        for rounding in (0, 1, 2):
+            c, s = gpu.mxfp4_transform_quantize(_dev(x), reduce_dim, _dev(Qb), seed, 5, rounding, gpu.SF_LINEAR)
+            rc, rs = ref.quantize(y_gpu, rounding, seed, 5)
+            assert np.array_equal(hp.unpack_codes(c.cpu().numpy()), rc)
+            assert np.array_equal(s.cpu().numpy().reshape(R, K // 32), rs)
+    assert gpu.mxfp4_device_status() == 0
