@@ -31,16 +31,6 @@ __device__ __forceinline__ uint32_t smem_u32(const void* p) {
     return static_cast<uint32_t>(__cvta_generic_to_shared(p));
 }
 
-__device__ __forceinline__ bool elect_one() {
-    uint32_t pred;
-    asm volatile(
-        "{\n\t.reg .pred p;\n\t"
-        "elect.sync _|p, 0xffffffff;\n\t"
-        "selp.u32 %0, 1, 0, p;\n\t}"
-        : "=r"(pred));
-    return pred != 0;
-}
-
 // Programmatic dependent launch: a kernel launched with the programmatic-serialisation attribute may start while
 // its predecessor in the stream is still running.  pdl_launch_dependents lets the successor's CTAs be scheduled as
 // soon as resources free up; pdl_wait blocks until the predecessor grid has completed and its writes are visible
@@ -196,13 +186,8 @@ __device__ __forceinline__ uint64_t make_smem_desc(uint32_t saddr, uint32_t lbo_
            (1ull << 46) | ((uint64_t)swizzle << 61);
 }
 
-// Copy 32 rows x 16 bytes of scale factors from shared memory to 4 TMEM columns, replicated to the four
-// 32-lane quadrants.
-__device__ __forceinline__ void tc_cp_32x128b_warpx4(uint32_t taddr, uint64_t sdesc) {
-    asm volatile("tcgen05.cp.cta_group::1.32x128b.warpx4 [%0], %1;" ::"r"(taddr), "l"(sdesc) : "memory");
-}
-
-// The same copy issued for a CTA pair: each CTA's copy reads its own shared memory and writes its own TMEM.
+// Copy 32 rows x 16 bytes of scale factors from shared memory to 4 TMEM columns, replicated to the four 32-lane
+// quadrants, issued for a CTA pair: each CTA's copy reads its own shared memory and writes its own TMEM.
 __device__ __forceinline__ void tc_cp_32x128b_warpx4_pair(uint32_t taddr, uint64_t sdesc) {
     asm volatile("tcgen05.cp.cta_group::2.32x128b.warpx4 [%0], %1;" ::"r"(taddr), "l"(sdesc) : "memory");
 }
