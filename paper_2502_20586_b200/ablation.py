@@ -3,8 +3,8 @@
     python -m paper_2502_20586_b200.ablation [--M 16384 --N 8192 --K 2048] [--json out.json]
 
 C = A B^T with a gradient-like A [M, K] (Student-t, std 1e-4, outlier rate in {0, 0.1 %, 1 %} at x50) and a
-weight-like B [N, K] (N(0, 0.02^2)), reduce K.  For g in {32, 64, 128, 256} and the four modes
-{RHT + SR, SR only, RHT + nearest, nearest} it reports the relative Frobenius error of the MXFP4 product against the
+weight-like B [N, K] (N(0, 0.02^2)), reduce K.  For g in {32, 64, 128, 256} and the modes
+{RHT + SR, SR only, RHT + nearest, nearest, RHT + SR with the 16-bit dither} it reports the relative Frobenius error of the MXFP4 product against the
 fp64 product of the bf16 inputs, and the throughput of quantise(A) + quantise(B) + GEMM.  Without the RHT the block
 size g has no effect; those cells are repeated so the table is complete.
 """
@@ -36,7 +36,8 @@ def mxfp4_product(A, B, g, rounding, seed, out=None):
     return mx.mxfp4_gemm(ca, sa, cb, sb, 16.0 / 9.0 if rounding != mx.ROUND_RN else 1.0, mx.OUT_FP32, C_out=out)
 
 
-MODES = (("RHT+SR", True, mx.ROUND_SR), ("SR", False, mx.ROUND_SR), ("RHT+RN", True, mx.ROUND_RN), ("RN", False, mx.ROUND_RN))
+MODES = (("RHT+SR", True, mx.ROUND_SR), ("SR", False, mx.ROUND_SR), ("RHT+RN", True, mx.ROUND_RN), ("RN", False, mx.ROUND_RN),
+         ("RHT+SR16", True, mx.ROUND_SR16))          # the last: the 16-bit-dither reading of SR (hardware convert)
 
 
 def run(M, N, K, rates=(0.0, 1e-3, 1e-2), gs=(32, 64, 128, 256), seed=0, iters=5):
@@ -76,13 +77,13 @@ def main():
     args = ap.parse_args()
     rows = run(args.M, args.N, args.K)
     print(f"# C = A B^T, M={args.M} N={args.N} K={args.K}; relative Frobenius error vs fp64 product of the bf16 inputs")
-    print("| outlier rate | g | " + " | ".join(m[0] for m in MODES) + " | TFLOP/s incl. quantise (RHT+SR) |")
-    print("|---|---|" + "---|" * (len(MODES) + 1))
+    print("| outlier rate | g | " + " | ".join(m[0] for m in MODES) + " | TFLOP/s incl. quantise (RHT+SR) | (RHT+SR16) | (RN, no RHT) |")
+    print("|---|---|" + "---|" * (len(MODES) + 3))
     for rate in sorted({r["outlier_rate"] for r in rows}):
         for g in sorted({r["g"] for r in rows}):
             cell = {r["mode"]: r for r in rows if r["outlier_rate"] == rate and r["g"] == g}
             print(f"| {rate:g} | {g} | " + " | ".join(f"{cell[m[0]]['rel_error']:.4f}" for m in MODES) +
-                  f" | {cell['RHT+SR']['tflops_incl_quantize']:.0f} |")
+                  f" | {cell['RHT+SR']['tflops_incl_quantize']:.0f} | {cell['RHT+SR16']['tflops_incl_quantize']:.0f} | {cell['RN']['tflops_incl_quantize']:.0f} |")
     if args.json:
         with open(args.json, "w") as fh:
             json.dump(rows, fh, indent=1)

@@ -1,4 +1,4 @@
-"""Error ablation on one GEMM (the g x {RHT+SR, SR, RHT+RN, RN} sweep), checked against the oracle on a reduced shape."""
+"""Error ablation on one GEMM (the g x {RHT+SR, SR, RHT+RN, RN, RHT+SR16} sweep), checked against the oracle on a reduced shape."""
 import numpy as np
 import pytest
 
@@ -24,7 +24,7 @@ def test_ablation_errors_match_oracle_and_have_the_expected_order(ref):
             C = ablation.mxfp4_product(dev(A), dev(B), geff, rounding, 5).cpu().numpy().astype(np.float64)
             _, ca, sa = ref.rht_quantize(A, geff, rounding, 5, 1)
             _, cb, sb = ref.rht_quantize(B, geff, rounding, 5, 2)
-            Co = ref.gemm(ca, sa, cb, sb, alpha=16 / 9 if rounding == ref.ROUND_SR else 1.0)
+            Co = ref.gemm(ca, sa, cb, sb, alpha=16 / 9 if rounding != ref.ROUND_RN else 1.0)
             e_gpu = np.linalg.norm(C - exact) / np.linalg.norm(exact)
             e_ora = np.linalg.norm(Co - exact) / np.linalg.norm(exact)
             assert abs(e_gpu - e_ora) <= 0.02 * e_ora + 1e-4, (g, name, e_gpu, e_ora)
@@ -35,3 +35,4 @@ def test_ablation_errors_match_oracle_and_have_the_expected_order(ref):
         assert errs[(g, "RHT+SR")] < errs[(g, "SR")]
         assert errs[(g, "RN")] < errs[(g, "SR")]                  # SR buys unbiasedness, not one-shot error
         assert 0.03 < errs[(g, "RHT+SR")] < 0.6
+        assert abs(errs[(g, "RHT+SR16")] - errs[(g, "RHT+SR")]) < 0.1 * errs[(g, "RHT+SR")]     # the two SR readings differ only in their noise
