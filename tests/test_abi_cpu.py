@@ -145,3 +145,15 @@ def test_binding_fails_loudly_without_library(tmp_path, monkeypatch):
     mod = importlib.util.module_from_spec(spec)
     with pytest.raises(ImportError):
         spec.loader.exec_module(mod)
+
+
+def test_header_is_plain_c(tmp_path):
+    """The boundary is a C ABI: include/mxfp4.h compiles as C99 and as C++ with nothing but the standard headers."""
+    import shutil
+    import subprocess
+    if shutil.which("gcc") is None:
+        pytest.skip("no gcc")
+    src = tmp_path / "use_header.c"
+    src.write_text('#include "include/mxfp4.h"\nint main(void) { return (int)MXFP4_ROUND_SR16 + (int)MXFP4_ERR_TIMEOUT; }\n')
+    for cmd in (["gcc", "-std=c99", "-Wall", "-Wextra", "-pedantic", "-Werror"], ["g++", "-std=c++11", "-Wall", "-Wextra", "-Werror", "-x", "c++"]):
+        subprocess.run(cmd + ["-I", ROOT, "-fsyntax-only", str(src)], check=True)
