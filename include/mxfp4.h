@@ -238,6 +238,14 @@ MXFP4_API mxfp4_status mxfp4_linear_backward_static(const void* dY, const void* 
  */
 MXFP4_API mxfp4_status mxfp4_fp4_ceiling(int64_t mma_per_pair, int64_t* flop_out, void* cuda_stream);
 
+/*
+ * Diagnostic, not part of the method: launches one warp that waits on a barrier nothing signals.  Every device-side
+ * wait of the library is bounded (about two seconds); when one expires the kernel records a status word, unwinds and
+ * returns normally.  This call takes exactly that path without any fault: after it, mxfp4_device_status returns
+ * MXFP4_ERR_TIMEOUT once (and clears the word), and the context stays usable.  Takes about two seconds of device time.
+ */
+MXFP4_API mxfp4_status mxfp4_selftest_wait_expiry(void* cuda_stream);
+
 /* Size in bytes of a scale tensor for an operand [rows, K] in the given layout (NATIVE is padded). */
 MXFP4_API size_t mxfp4_scale_bytes(int64_t rows, int64_t K, int sf_layout);
 

@@ -47,6 +47,8 @@ _lib.mxfp4_operand_layout.argtypes = [_i64, _i64, _i64, C.POINTER(_sz)]
 _lib.mxfp4_operand_layout.restype = None
 _lib.mxfp4_quantize_operands.argtypes = [_vp, _vp, _vp, _i64, _i64, _i64, _int, _int, _u64, _vp, _sz, _vp]
 _lib.mxfp4_quantize_operands.restype = _int
+_lib.mxfp4_selftest_wait_expiry.argtypes = [_vp]
+_lib.mxfp4_selftest_wait_expiry.restype = _int
 _lib.mxfp4_fp4_ceiling.argtypes = [_i64, C.POINTER(C.c_int64), _vp]
 _lib.mxfp4_fp4_ceiling.restype = _int
 _lib.mxfp4_scale_bytes.argtypes = [_i64, _i64, _int]
@@ -59,7 +61,8 @@ _lib.mxfp4_status_string.restype = C.c_char_p
 EXPORTS = ["mxfp4_rht_sr_quantize", "mxfp4_rht", "mxfp4_gemm", "mxfp4_linear_backward_workspace",
            "mxfp4_linear_backward", "mxfp4_linear_backward_static", "mxfp4_scale_bytes", "mxfp4_device_status", "mxfp4_status_string",
            "mxfp4_fp4_ceiling", "mxfp4_linear_backward_ex_workspace", "mxfp4_linear_backward_ex", "mxfp4_gemm_fused",
-           "mxfp4_linear_backward_fused", "mxfp4_operand_layout", "mxfp4_quantize_operands", "mxfp4_transform_quantize"]
+           "mxfp4_linear_backward_fused", "mxfp4_operand_layout", "mxfp4_quantize_operands", "mxfp4_transform_quantize",
+           "mxfp4_selftest_wait_expiry"]
 
 
 class MxFp4Error(RuntimeError):
@@ -84,6 +87,11 @@ def _ptr(t) -> int:
 def lib():
     """The raw ctypes handle (tests use it to probe error codes with arbitrary arguments)."""
     return _lib
+
+
+def mxfp4_selftest_wait_expiry() -> None:
+    """Launch the diagnostic kernel whose bounded wait expires (about two seconds); the next device status is TIMEOUT."""
+    _check(_lib.mxfp4_selftest_wait_expiry(_stream()))
 
 
 def mxfp4_scale_bytes(rows: int, K: int, sf_layout: int = SF_NATIVE) -> int:

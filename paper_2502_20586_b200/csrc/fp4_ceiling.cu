@@ -91,11 +91,32 @@ fp4_ceiling_kernel(uint32_t batches) {
     }
 }
 
+// Diagnostic: one thread waits on a barrier that nothing ever signals.  The bounded wait gives up after its time limit,
+// records the status word and the kernel returns normally: the path every kernel of the library takes when a wait
+// expires, exercised without a fault.
+__global__ void wait_expiry_kernel() {
+    __shared__ uint64_t bar;
+    if (threadIdx.x == 0) {
+        mbar_init(&bar, 1);
+        mbar_fence_init();
+        (void)mbar_wait(&bar, 0);            // phase 0 never completes: returns false after the limit, status word set
+    }
+}
+
 }  // namespace
 
 cudaError_t fetch_fp4_ceiling_status(unsigned int* word) { return device_status_fetch(word); }
 
 }  // namespace mx
+
+extern "C" mxfp4_status mxfp4_selftest_wait_expiry(void* cuda_stream) {
+    int dev = 0, major = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess || cudaDeviceGetAttribute(&major, cudaDevAttrComputeCapabilityMajor, dev) != cudaSuccess)
+        return MXFP4_ERR_CUDA;
+    if (major != 10) return MXFP4_ERR_DEVICE;
+    mx::wait_expiry_kernel<<<1, 32, 0, static_cast<cudaStream_t>(cuda_stream)>>>();
+    return cudaGetLastError() == cudaSuccess ? MXFP4_OK : MXFP4_ERR_CUDA;
+}
 
 extern "C" mxfp4_status mxfp4_fp4_ceiling(int64_t mma_per_pair, int64_t* flop_out, void* cuda_stream) {
     if (mma_per_pair <= 0 || flop_out == nullptr) return MXFP4_ERR_SHAPE;
