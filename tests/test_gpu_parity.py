@@ -358,8 +358,8 @@ def test_split_form_equals_the_one_call_form(gpu):
     dY = (torch.randn(b, m, device="cuda", generator=gen) * 1e-3).to(torch.bfloat16)
     X = torch.randn(b, n, device="cuda", generator=gen).to(torch.bfloat16)
     W = (torch.randn(m, n, device="cuda", generator=gen) * 0.02).to(torch.bfloat16)
-    for rounding, alpha in ((gpu.ROUND_SR, 16 / 9), (gpu.ROUND_RN, 1.0), (gpu.ROUND_SR16, 16 / 9)):
-        q = gpu.mxfp4_quantize_operands(dY, X, W, g, 17, rounding)
+    for rounding, alpha, g in ((gpu.ROUND_SR, 16 / 9, 128), (gpu.ROUND_RN, 1.0, 128), (gpu.ROUND_SR16, 16 / 9, 128), (gpu.ROUND_SR, 16 / 9, 0)):
+        q = gpu.mxfp4_quantize_operands(dY, X, W, g, 17, rounding)      # g = 0: the views go through the CUDA-core quantiser one by one
         dX = gpu.mxfp4_gemm(q[0][0], q[0][1], q[1][0], q[1][1], alpha, gpu.OUT_FP32)
         dW = gpu.mxfp4_gemm(q[2][0], q[2][1], q[3][0], q[3][1], alpha, gpu.OUT_FP32)
         rX, rW = gpu.mxfp4_linear_backward(dY, X, W, g, 17, rounding, gpu.OUT_FP32)
