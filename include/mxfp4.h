@@ -18,8 +18,13 @@
  *     legacy default stream).
  *   - Tensors are row-major.  bf16 data, codes and scales must be 16-byte
  *     aligned; leading dimensions must keep every row 16-byte aligned.
- *   - Return value: MXFP4_OK or an error code; on error nothing was enqueued.
- *     Invalid arguments are reported as errors, never as undefined behaviour.
+ *   - Return value: MXFP4_OK or an error code.  Invalid arguments are reported
+ *     as errors, never as undefined behaviour, and every argument check and
+ *     tensor-map encoding happens before the first launch: for all codes
+ *     except MXFP4_ERR_CUDA nothing was enqueued.  MXFP4_ERR_CUDA may come from
+ *     a kernel launch the driver refused after earlier kernels of the same call
+ *     were enqueued; outputs are then undefined, but the stream stays ordered
+ *     (a call that used its side stream has joined it back).
  *   - Inputs must be finite.  A block containing Inf/NaN gets scale byte 255.
  *   - Same inputs + same seed => bit-identical outputs.
  */
@@ -219,7 +224,10 @@ MXFP4_API mxfp4_status mxfp4_linear_backward_fused(const void* dY, const void* X
  *   MXFP4_ERR_WORKSPACE; nothing is enqueued.
  *   The call allocates nothing, neither on the host nor on the device.
  *   The first call on each device looks up the array's device address (cudaGetSymbolAddress, with that device
- *   current); make that first call outside any stream capture.
+ *   current); make that first call outside any stream capture.  That first call is also the moment at which the
+ *   CUDA runtime may load the library's kernels and the array itself onto the device (module loading is lazy), which
+ *   does need free device memory: a caller that wants the call to survive memory exhaustion makes one warm-up call
+ *   per device while memory is still available.  Later calls take nothing from any allocator.
  *   All calls on a device share the one array, which keeps whatever the previous call left in it.  Each call rewrites
  *   every byte it later reads, so nothing needs clearing between calls; but two calls whose kernels can overlap on
  *   the GPU (different streams without ordering) race on it: order them.
@@ -234,8 +242,11 @@ MXFP4_API mxfp4_status mxfp4_linear_backward_static(const void* dY, const void* 
  * issues `mma_per_pair` (rounded up to a multiple of 32) back-to-back 256 x 256 x 64 block-scaled FP4 tensor-core
  * instructions on operands resident in shared memory: no loads, no output.  *flop_out (HOST pointer) receives the
  * floating-point operations the launch performs; time the launch with CUDA events on `cuda_stream` to obtain the
- * on-box ceiling of the FP4 tensor pipe.  Errors: MXFP4_ERR_SHAPE, MXFP4_ERR_DEVICE, MXFP4_ERR_CUDA.
+ * on-box ceiling of the FP4 tensor pipe.  mma_per_pair is limited to MXFP4_CEILING_MAX_MMA_PER_PAIR (about two seconds
+ * of device time: the kernel cannot be stopped once launched); larger values are refused with MXFP4_ERR_SHAPE.
+ * Errors: MXFP4_ERR_SHAPE, MXFP4_ERR_DEVICE, MXFP4_ERR_CUDA.
  */
+#define MXFP4_CEILING_MAX_MMA_PER_PAIR 20000000
 MXFP4_API mxfp4_status mxfp4_fp4_ceiling(int64_t mma_per_pair, int64_t* flop_out, void* cuda_stream);
 
 /*

@@ -211,6 +211,13 @@ def mxfp4_quantize_operands(dY, X, W, g: int, seed: int, rounding: int = ROUND_S
     return out
 
 
+def mxfp4_operand_layout(b: int, m: int, n: int):
+    """Byte offsets [(codes, scales)] x 4 of the quantised operands Q1..Q4 inside a backward workspace."""
+    off = (_sz * 8)()
+    _lib.mxfp4_operand_layout(b, m, n, off)
+    return [(int(off[2 * i]), int(off[2 * i + 1])) for i in range(4)]
+
+
 def mxfp4_linear_backward_workspace(b: int, m: int, n: int) -> int:
     return int(_lib.mxfp4_linear_backward_workspace(b, m, n))
 

@@ -157,10 +157,9 @@ bool make_output_map(CUtensorMap* map, void* C, int64_t M, int64_t N, int64_t ld
     return r == CUDA_SUCCESS;
 }
 
-mxfp4_status gemm_impl(const uint8_t* A_codes, const uint8_t* A_scales, const uint8_t* B_codes, const uint8_t* B_scales, int64_t M,
-                       int64_t N, int64_t K, float alpha, void* C, int64_t ldc, int out_dtype, cudaStream_t stream,
-                       int accumulate = 0) {
-    GemmArgs a;
+// Everything a GEMM launch needs (tensor maps included), built without touching the device.
+mxfp4_status gemm_prepare(GemmArgs& a, const uint8_t* A_codes, const uint8_t* A_scales, const uint8_t* B_codes, const uint8_t* B_scales,
+                          int64_t M, int64_t N, int64_t K, float alpha, void* C, int64_t ldc, int out_dtype, int accumulate) {
     mxfp4_status st = make_codes_map(&a.tmap_a, A_codes, M, K, mx::kGemmBM);
     if (st != MXFP4_OK) return st;
     st = make_codes_map(&a.tmap_b, B_codes, N, K, mx::kGemmBN);
@@ -170,13 +169,26 @@ mxfp4_status gemm_impl(const uint8_t* A_codes, const uint8_t* A_scales, const ui
     a.alpha = alpha; a.C = C; a.ldc = ldc; a.out_fp32 = out_dtype == MXFP4_OUT_FP32;
     a.accumulate = accumulate;
     a.use_pair = g_rt.gemm_pair && M > 128;                   // one 128-row tile gives a pair nothing to share
+    a.has_tmap_c = false;
     if (a.use_pair) {
         st = make_codes_map(&a.tmap_b_half, B_codes, N, K, 128);
         if (st != MXFP4_OK) return st;
         a.has_tmap_c = make_output_map(&a.tmap_c, C, M, N, ldc, a.out_fp32 != 0);
-        return mx::launch_gemm_pair(a, stream) == cudaSuccess ? MXFP4_OK : MXFP4_ERR_CUDA;
     }
-    return mx::launch_gemm(a, stream) == cudaSuccess ? MXFP4_OK : MXFP4_ERR_CUDA;
+    return MXFP4_OK;
+}
+
+mxfp4_status gemm_launch(const GemmArgs& a, cudaStream_t stream) {
+    const cudaError_t e = a.use_pair ? mx::launch_gemm_pair(a, stream) : mx::launch_gemm(a, stream);
+    return e == cudaSuccess ? MXFP4_OK : MXFP4_ERR_CUDA;
+}
+
+mxfp4_status gemm_impl(const uint8_t* A_codes, const uint8_t* A_scales, const uint8_t* B_codes, const uint8_t* B_scales, int64_t M,
+                       int64_t N, int64_t K, float alpha, void* C, int64_t ldc, int out_dtype, cudaStream_t stream,
+                       int accumulate = 0) {
+    GemmArgs a;
+    const mxfp4_status st = gemm_prepare(a, A_codes, A_scales, B_codes, B_scales, M, N, K, alpha, C, ldc, out_dtype, accumulate);
+    return st != MXFP4_OK ? st : gemm_launch(a, stream);
 }
 
 // C = alpha Q(RHT(A)) deq(B)^T with A = x (reduce_dim 1) or x^T (reduce_dim 0) quantised inside the GEMM kernel.
@@ -377,24 +389,28 @@ mxfp4_status linear_backward_impl(const void* dY, const void* X, const void* W, 
     uint8_t* base = static_cast<uint8_t*>(workspace);
     uint8_t *c[4], *s[4];
     for (int i = 0; i < 4; ++i) { c[i] = base + ws.codes[i]; s[i] = base + ws.scales[i]; }
-    if ((st = quantize_operands_impl(dY, X, W, b, m, n, g, rounding, seed, c, s, stream)) != MXFP4_OK) return st;
     // lines 7-11: two MXFP4 GEMMs; the 16/9 un-does the two 3/4 pre-scales of Algorithm 2.
     const float alpha = rounding != MXFP4_ROUND_RN ? 16.0f / 9.0f : 1.0f;       // both SR modes carry the 3/4 pre-scale
+    // Every tensor map is encoded before the first launch, so an encoding failure leaves nothing enqueued.
+    GemmArgs gx, gw;
+    if ((st = gemm_prepare(gx, c[0], s[0], c[1], s[1], b, n, m, alpha, dX, n, out_dtype, 0)) != MXFP4_OK) return st;   // dX is never accumulated
+    if ((st = gemm_prepare(gw, c[2], s[2], c[3], s[3], m, n, b, alpha, dW, n, out_dtype, accumulate)) != MXFP4_OK) return st;
+    if ((st = quantize_operands_impl(dY, X, W, b, m, n, g, rounding, seed, c, s, stream)) != MXFP4_OK) return st;
     // Large problems (never the ones the fixed-scratch variant accepts) run the two GEMMs fork / join.
     const int64_t waves_dx = ((b + 255) / 256) * ((n + 255) / 256), waves_dw = ((m + 255) / 256) * ((n + 255) / 256);
     ForkJoin* fj = ws.total > (size_t)MXFP4_STATIC_WORKSPACE_BYTES && waves_dx >= 74 && waves_dw >= 74 ? fork_join() : nullptr;
     if (fj != nullptr && (cudaEventRecord(fj->fork, stream) != cudaSuccess || cudaStreamWaitEvent(fj->side, fj->fork, 0) != cudaSuccess))
-        return MXFP4_ERR_CUDA;
-    st = gemm_impl(c[0], s[0], c[1], s[1], b, n, m, alpha, dX, n, out_dtype, stream);      // dX is never accumulated
-    if (st != MXFP4_OK) return st;
-    st = gemm_impl(c[2], s[2], c[3], s[3], m, n, b, alpha, dW, n, out_dtype, fj != nullptr ? fj->side : stream, accumulate);
-    if (st != MXFP4_OK) return st;
+        fj = nullptr;                                // the side stream was not given anything yet: stay on the caller's stream
+    st = gemm_launch(gx, stream);
+    if (st == MXFP4_OK) st = gemm_launch(gw, fj != nullptr ? fj->side : stream);
     // dL/db = 1 dL/dy (problem statement): column sums of dY, after the GEMMs on the caller's stream
-    if (db != nullptr && mx::launch_bias_grad(dY, b, m, m, accumulate, db, reinterpret_cast<float*>(base + bias_off), stream) != cudaSuccess)
-        return MXFP4_ERR_CUDA;
+    if (st == MXFP4_OK && db != nullptr &&
+        mx::launch_bias_grad(dY, b, m, m, accumulate, db, reinterpret_cast<float*>(base + bias_off), stream) != cudaSuccess)
+        st = MXFP4_ERR_CUDA;
+    // The join is made whatever happened after the fork, so that the side stream never runs unordered with the caller's.
     if (fj != nullptr && (cudaEventRecord(fj->join, fj->side) != cudaSuccess || cudaStreamWaitEvent(stream, fj->join, 0) != cudaSuccess))
         return MXFP4_ERR_CUDA;
-    return MXFP4_OK;
+    return st;
 }
 }  // namespace
 

@@ -119,7 +119,8 @@ extern "C" mxfp4_status mxfp4_selftest_wait_expiry(void* cuda_stream) {
 }
 
 extern "C" mxfp4_status mxfp4_fp4_ceiling(int64_t mma_per_pair, int64_t* flop_out, void* cuda_stream) {
-    if (mma_per_pair <= 0 || flop_out == nullptr) return MXFP4_ERR_SHAPE;
+    // 2e7 instructions per pair are about two seconds of device time: the kernel cannot be pre-empted or stopped early
+    if (mma_per_pair <= 0 || mma_per_pair > MXFP4_CEILING_MAX_MMA_PER_PAIR || flop_out == nullptr) return MXFP4_ERR_SHAPE;
     int dev = 0, sms = 0, major = 0;
     if (cudaGetDevice(&dev) != cudaSuccess || cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess ||
         cudaDeviceGetAttribute(&major, cudaDevAttrComputeCapabilityMajor, dev) != cudaSuccess)

@@ -133,6 +133,7 @@ def test_argument_validation_needs_no_device(lib):
     # measurement aid
     assert raw.mxfp4_fp4_ceiling(0, C.byref(C.c_int64(0)), 0) == 2
     assert raw.mxfp4_fp4_ceiling(64, None, 0) == 2
+    assert raw.mxfp4_fp4_ceiling(20000001, C.byref(C.c_int64(0)), 0) == 2      # beyond the documented cap (about two seconds of device time)
 
 
 def test_binding_fails_loudly_without_library(tmp_path, monkeypatch):

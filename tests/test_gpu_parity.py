@@ -111,12 +111,8 @@ def test_quantizer_end_to_end_mismatch_rate(gpu, ref, g, rounding):
         x = _inputs("act", shape, 5)
         codes, scales = _quant_gpu(gpu, x, reduce_dim, g, 99, 1, rounding, gpu.SF_NATIVE)
         _, rc, rs = ref.rht_quantize(x, g, rounding, 99, 1, transpose=(reduce_dim == 0))
-        same_scale = (scales == rs).repeat(32, axis=1)
         assert (scales != rs).mean() <= 1e-5                      # amax within rounding of a power of two
-        diff = (codes != rc) & same_scale
-        assert diff.mean() <= 1e-4
-        step = np.abs(hp.E2M1_STEP_INDEX[codes[diff]] - hp.E2M1_STEP_INDEX[rc[diff]])
-        assert np.all(step <= 1)
+        hp.compare_quantised_rows(codes, scales, rc, rs)          # such blocks are compared by their dequantised values
 
 
 @pytest.mark.parametrize("rounding", [0, 2])
@@ -236,14 +232,17 @@ def test_linear_backward_single_layer(gpu, ref, rounding):
     assert gpu.mxfp4_device_status() == 0
     dX = dX.cpu().numpy().astype(np.float64); dW = dW.cpu().numpy().astype(np.float64)
     rdX, rdW = ref.linear_backward(dY, X, W, 64, rounding, 0)
-    # codes may differ in <= 1e-4 of the elements by one step, so the end-to-end outputs agree closely, not bitwise
-    assert np.linalg.norm(dX - rdX) / np.linalg.norm(rdX) <= 2e-2
-    assert np.linalg.norm(dW - rdW) / np.linalg.norm(rdW) <= 2e-2
     # strict: the GEMMs reproduce the fp64 product of the operands the GPU itself quantised
     tags = {1: (dY, 1), 2: (W, 0), 3: (dY, 0), 4: (X, 0)}
-    q = {}
+    q, rate = {}, {}
     for tag, (t, rd) in tags.items():
         q[tag] = _quant_gpu(gpu, t, rd, 64, 0, tag, rounding, gpu.SF_NATIVE)
+        _, oc, os_ = ref.rht_quantize(t, 64, rounding, 0, tag, transpose=(rd == 0))
+        rate[tag] = hp.compare_quantised_rows(q[tag][0], q[tag][1], oc, os_)
+    # codes may differ in <= 1e-4 of the elements by one step, so the end-to-end outputs agree closely, not bitwise:
+    # the bound follows from the differences actually counted (1e-5 when there are none)
+    assert np.linalg.norm(dX - rdX) / np.linalg.norm(rdX) <= hp.product_tolerance(rate[1], rate[2])
+    assert np.linalg.norm(dW - rdW) / np.linalg.norm(rdW) <= hp.product_tolerance(rate[3], rate[4])
     alpha = 16 / 9 if rounding != 1 else 1.0
     assert np.linalg.norm(dX - ref.gemm(*q[1], *q[2], alpha=alpha)) / np.linalg.norm(rdX) <= 1e-5
     assert np.linalg.norm(dW - ref.gemm(*q[3], *q[4], alpha=alpha)) / np.linalg.norm(rdW) <= 1e-5

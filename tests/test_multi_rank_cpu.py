@@ -3,9 +3,14 @@
 The backward path is data parallel over tokens with no exchange inside it, so bench.py --gpus N runs N replicas on
 their own tokens and combines only timings: whole-job FLOPs over the slowest rank's time.  This test drives that
 host-side logic (seeding per rank, max-over-ranks reduction, aggregate value) with world_size 2 on the gloo backend.
+The last test starts `python bench.py --gpus 2` the way a user would (no torchrun, no WORLD_SIZE): the script must
+launch the two ranks itself and report n_gpus = 2; a CPU stub of the step stands in for the GPU work.
 """
+import json
 import os
 import socket
+import subprocess
+import sys
 
 import pytest
 import torch
@@ -51,3 +56,18 @@ def test_single_rank_needs_no_process_group():
     import bench
     assert bench.max_over_ranks(1.5, None, 1, torch.device("cpu")) == (1.5, None)
     assert bench.aggregate_value(4e12, 1, 2.0) == pytest.approx(2000.0)
+
+
+def test_bench_gpus_flag_starts_the_ranks_itself():
+    root = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+    env = {k: v for k, v in os.environ.items() if k not in ("WORLD_SIZE", "RANK", "LOCAL_RANK", "MASTER_ADDR", "MASTER_PORT")}
+    out = subprocess.run([sys.executable, os.path.join(root, "bench.py"), "--gpus", "2", "--steps", "2", "--warmup", "1", "--stub-cpu"],
+                         env=env, capture_output=True, text=True, timeout=300)
+    assert out.returncode == 0, out.stderr[-2000:]
+    lines = [l for l in out.stdout.splitlines() if l.startswith("{")]
+    assert len(lines) == 1                                     # rank 0 alone prints
+    rec = json.loads(lines[0])
+    assert rec["n_gpus"] == 2
+    assert rec["ms_per_step"] == 5.0                           # the slower rank's time
+    assert rec["value"] == pytest.approx(2 * 6e12 / 5e-3 / 1e12)
+    assert rec["seeds"][0] != rec["seeds"][1]
