@@ -3,6 +3,7 @@
 #include <cuda_runtime.h>
 #include <stdint.h>
 
+#include <cstdio>
 #include <cstdlib>
 #include <mutex>
 
@@ -49,6 +50,14 @@ mxfp4_status runtime_init() {
     if (g_rt.status != MXFP4_OK) return g_rt.status;
     int dev = 0;
     if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= Runtime::kMaxDevices) return MXFP4_ERR_CUDA;
+    // Tensor-map encoding is a driver call and needs the device's context current on the CALLING thread.  A thread
+    // that has only inherited the device number (a framework's worker thread) may not have it bound yet: selecting the
+    // device it already names binds the primary context.  Done once per thread and device.
+    static thread_local int bound_dev = -1;
+    if (bound_dev != dev) {
+        if (cudaSetDevice(dev) != cudaSuccess) return MXFP4_ERR_CUDA;
+        bound_dev = dev;
+    }
     std::lock_guard<std::mutex> lock(g_rt.mu);
     if (!g_rt.dev_done[dev]) {
         int major = 0;
@@ -91,6 +100,19 @@ ForkJoin* fork_join() {
     return fj.ok && fj.device == dev ? &fj : nullptr;
 }
 
+// With MXFP4_DEBUG set in the environment a failing CUDA call is named on stderr (the ABI only returns MXFP4_ERR_CUDA).
+mxfp4_status cuda_status(cudaError_t e, const char* where) {
+    if (e == cudaSuccess) return MXFP4_OK;
+    if (getenv("MXFP4_DEBUG") != nullptr) fprintf(stderr, "mxfp4: %s failed: %s\n", where, cudaGetErrorString(e));
+    return MXFP4_ERR_CUDA;
+}
+
+mxfp4_status encode_status(CUresult r, const char* where) {
+    if (r == CUDA_SUCCESS) return MXFP4_OK;
+    if (getenv("MXFP4_DEBUG") != nullptr) fprintf(stderr, "mxfp4: tensor-map encoding failed (%s): CUresult %d\n", where, (int)r);
+    return MXFP4_ERR_CUDA;
+}
+
 bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
 bool valid_g(int g) { return g == 0 || g == 32 || g == 64 || g == 128 || g == 256; }
 int64_t round_up(int64_t v, int64_t a) { return (v + a - 1) / a * a; }
@@ -123,7 +145,9 @@ mxfp4_status make_codes_map(CUtensorMap* map, const uint8_t* codes, int64_t rows
     const CUresult r = g_rt.encode(map, CU_TENSOR_MAP_DATA_TYPE_UINT8, 2, const_cast<uint8_t*>(codes), dims, strides, box, elem_strides,
                                    CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
                                    CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
-    return r == CUDA_SUCCESS ? MXFP4_OK : MXFP4_ERR_CUDA;
+    if (r != CUDA_SUCCESS && getenv("MXFP4_DEBUG") != nullptr)
+        fprintf(stderr, "mxfp4: codes map: ptr %p rows %lld K %lld box_rows %d\n", (const void*)codes, (long long)rows, (long long)K, box_rows);
+    return encode_status(r, "codes");
 }
 
 // Tensor map over the bf16 input [rows, cols] (leading dimension ld): box = 64 columns x 128 rows, 128-byte swizzle.
@@ -179,8 +203,7 @@ mxfp4_status gemm_prepare(GemmArgs& a, const uint8_t* A_codes, const uint8_t* A_
 }
 
 mxfp4_status gemm_launch(const GemmArgs& a, cudaStream_t stream) {
-    const cudaError_t e = a.use_pair ? mx::launch_gemm_pair(a, stream) : mx::launch_gemm(a, stream);
-    return e == cudaSuccess ? MXFP4_OK : MXFP4_ERR_CUDA;
+    return cuda_status(a.use_pair ? mx::launch_gemm_pair(a, stream) : mx::launch_gemm(a, stream), a.use_pair ? "pair GEMM launch" : "GEMM launch");
 }
 
 mxfp4_status gemm_impl(const uint8_t* A_codes, const uint8_t* A_scales, const uint8_t* B_codes, const uint8_t* B_scales, int64_t M,
@@ -347,9 +370,9 @@ mxfp4_status quantize_operands_impl(const void* dY, const void* X, const void* W
         all_tc = all_tc && mx::quant_tc_eligible(q[i]);
     }
     if (all_tc)                                     // the four views of the call in one launch
-        return mx::launch_quantize_tc_group(q, 4, false, stream) == cudaSuccess ? MXFP4_OK : MXFP4_ERR_CUDA;
+        return cuda_status(mx::launch_quantize_tc_group(q, 4, false, stream), "grouped quantiser launch");
     for (int i = 0; i < 4; ++i)
-        if (mx::launch_quantize(q[i], stream) != cudaSuccess) return MXFP4_ERR_CUDA;
+        if (cuda_status(mx::launch_quantize(q[i], stream), "quantiser launch") != MXFP4_OK) return MXFP4_ERR_CUDA;
     return MXFP4_OK;
 }
 
@@ -404,9 +427,8 @@ mxfp4_status linear_backward_impl(const void* dY, const void* X, const void* W, 
     st = gemm_launch(gx, stream);
     if (st == MXFP4_OK) st = gemm_launch(gw, fj != nullptr ? fj->side : stream);
     // dL/db = 1 dL/dy (problem statement): column sums of dY, after the GEMMs on the caller's stream
-    if (st == MXFP4_OK && db != nullptr &&
-        mx::launch_bias_grad(dY, b, m, m, accumulate, db, reinterpret_cast<float*>(base + bias_off), stream) != cudaSuccess)
-        st = MXFP4_ERR_CUDA;
+    if (st == MXFP4_OK && db != nullptr)
+        st = cuda_status(mx::launch_bias_grad(dY, b, m, m, accumulate, db, reinterpret_cast<float*>(base + bias_off), stream), "bias gradient launch");
     // The join is made whatever happened after the fork, so that the side stream never runs unordered with the caller's.
     if (fj != nullptr && (cudaEventRecord(fj->join, fj->side) != cudaSuccess || cudaStreamWaitEvent(stream, fj->join, 0) != cudaSuccess))
         return MXFP4_ERR_CUDA;

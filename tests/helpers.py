@@ -75,8 +75,8 @@ def product_tolerance(rate_a: float, rate_b: float, out_bits: int = 24) -> float
     """Relative Frobenius bound between two MXFP4 products whose operands differ in the given fractions of elements,
     each by at most one grid step: a differing element changes its term by at most about the term's own size, so
     with zero-mean terms the relative change of a sum is about sqrt(rate); 4 is head-room.  Plus the GEMM's own
-    1e-5 and half an ulp of the output format (8 significand bits for bf16)."""
-    return 4.0 * np.sqrt(rate_a + rate_b) + 1e-5 + (2.0 ** -9 if out_bits == 8 else 0.0)
+    1e-5 and the unit roundoff of the output format (2^-8 for bf16's 8 significand bits)."""
+    return 4.0 * np.sqrt(rate_a + rate_b) + 1e-5 + (2.0 ** -8 if out_bits == 8 else 0.0)
 
 
 def band_rows(n_rows: int) -> np.ndarray:

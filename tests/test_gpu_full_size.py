@@ -99,7 +99,7 @@ def test_sampled_parity_at_full_shapes(ref, config, layer_name, rounding):
     bx = dX[It][:, Jt].float().cpu().numpy().astype(np.float64); bw = dW[Pt][:, Qt].float().cpu().numpy().astype(np.float64)
     assert np.linalg.norm(bx - ox) <= hp.product_tolerance(rate[1], rate[2], out_bits=8) * np.linalg.norm(ox)
     assert np.linalg.norm(bw - ow) <= hp.product_tolerance(rate[3], rate[4], out_bits=8) * np.linalg.norm(ow)
-    # against the product of the GPU's own codes only bf16 rounding is left, entry by entry (half an ulp = 2^-9)
+    # against the product of the GPU's own codes only bf16 rounding is left, entry by entry (unit roundoff 2^-8)
     assert np.all(np.abs(bx - rx) <= 2.0 ** -8 * np.abs(rx) + 1e-5 * np.sqrt(np.mean(rx ** 2)))
     assert np.all(np.abs(bw - rw) <= 2.0 ** -8 * np.abs(rw) + 1e-5 * np.sqrt(np.mean(rw ** 2)))
     # and it is a sane estimate of the true gradient entries (fp64 product of the bf16 inputs)
