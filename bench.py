@@ -354,6 +354,27 @@ def run_gpu(args):
             ms_var = a.elapsed_time(b) / k_var
             variants[other] = {"ms_per_step": ms_var, "value": flops_step / (ms_var * 1e-3) / 1e12, "steps": k_var,
                                "note": "this rank's step with the other SR reading (8-bit centred dither / 16-bit dither of the hardware convert), timed right after the main steps; compare runs with --rounding for a like-for-like number"}
+        # the overlapped form of the call (MXFP4_OVERLAP=1): the second product's operands are quantised on the same SMs
+        # while the first product's GEMM runs (small builds of both kernels share an SM); same outputs, alternating A/B
+        if g in (32, 64, 128):
+            ab = {"0": [], "1": []}
+            for rep in range(3):
+                for ov in ("0", "1"):
+                    os.environ["MXFP4_OVERLAP"] = ov
+                    step()
+                    a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+                    k_var = max(1, min(args.steps, 10))
+                    torch.cuda.synchronize()
+                    a.record(stream)
+                    for _ in range(k_var):
+                        step()
+                    b.record(stream)
+                    torch.cuda.synchronize()
+                    ab[ov].append(a.elapsed_time(b) / k_var)
+            os.environ.pop("MXFP4_OVERLAP", None)
+            ms_ser, ms_ovl = sorted(ab["0"])[1], sorted(ab["1"])[1]
+            variants["overlapped"] = {"ms_per_step": ms_ovl, "value": flops_step / (ms_ovl * 1e-3) / 1e12, "serial_ms_per_step_same_leg": ms_ser,
+                                      "steps": k_var, "note": "median of three alternating runs of the overlapped and the serial form; the default is the serial form"}
         # the fused-producer variant (dY transformed and rounded inside the GEMM kernels), a few steps: it is several times slower
         if g in (32, 64, 128) and all(l.b % 256 == 0 and l.m % 256 == 0 for l in layers):
             def step_fused():

@@ -113,6 +113,23 @@ mxfp4_status encode_status(CUresult r, const char* where) {
     return MXFP4_ERR_CUDA;
 }
 
+// MXFP4_OVERLAP: 0 (default) = serial form (quantise everything, then the two GEMMs); 1 = overlapped form with the
+// cheaper head first; 2 / 3 = overlapped with dX / dW first.  Read at every call so that one process can compare the
+// forms.  The overlapped form is off by default because it measured no faster (the GEMM runs at the board's power
+// limit, so quantiser work done beside it slows it by about the time that was hidden).
+// MXFP4_FORCE_LITE=1: every pair GEMM and every grouped quantiser launch uses the small build of its kernel (tests use
+// this to put the small builds through the ragged and tiny shapes that the overlapped form itself never sees).
+bool force_lite() {
+    const char* e = getenv("MXFP4_FORCE_LITE");
+    return e != nullptr && e[0] == '1';
+}
+
+int overlap_setting() {
+    const char* e = getenv("MXFP4_OVERLAP");
+    if (e == nullptr || e[0] == '\0') return 0;
+    return e[0] >= '0' && e[0] <= '3' ? e[0] - '0' : 0;
+}
+
 bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
 bool valid_g(int g) { return g == 0 || g == 32 || g == 64 || g == 128 || g == 256; }
 int64_t round_up(int64_t v, int64_t a) { return (v + a - 1) / a * a; }
@@ -194,6 +211,7 @@ mxfp4_status gemm_prepare(GemmArgs& a, const uint8_t* A_codes, const uint8_t* A_
     a.accumulate = accumulate;
     a.use_pair = g_rt.gemm_pair && M > 128;                   // one 128-row tile gives a pair nothing to share
     a.has_tmap_c = false;
+    a.lite = a.use_pair && force_lite();
     if (a.use_pair) {
         st = make_codes_map(&a.tmap_b_half, B_codes, N, K, 128);
         if (st != MXFP4_OK) return st;
@@ -356,8 +374,13 @@ size_t mxfp4_linear_backward_workspace(int64_t b, int64_t m, int64_t n) {
 
 namespace {
 // Algorithm 3 lines 3-6: the four operand views, stream tags 1..4, one sign vector (same seed) for all of them.
+struct Overlap {
+    int first;            // in: product to run first (0 = dX, 1 = dW), its operands are quantised up front; out: -1 if the call fell back to the serial form
+    ForkJoin* fj;
+    bool forked = false;  // the side stream holds work that the caller's stream has to wait for
+};
 mxfp4_status quantize_operands_impl(const void* dY, const void* X, const void* W, int64_t b, int64_t m, int64_t n, int g, int rounding,
-                                    uint64_t seed, uint8_t* const c[4], uint8_t* const s[4], cudaStream_t stream) {
+                                    uint64_t seed, uint8_t* const c[4], uint8_t* const s[4], cudaStream_t stream, Overlap* ov = nullptr) {
     QuantArgs q[4] = {
         {dY, b, m, m, 1, g, rounding, seed, 1u, c[0], s[0], 1, nullptr},   // dY   [b, K = m]
         {W, m, n, n, 0, g, rounding, seed, 2u, c[1], s[1], 1, nullptr},    // W^T  [n, K = m]
@@ -369,8 +392,23 @@ mxfp4_status quantize_operands_impl(const void* dY, const void* X, const void* W
         attach_input_map(q[i]);
         all_tc = all_tc && mx::quant_tc_eligible(q[i]);
     }
+    if (ov != nullptr && ov->first >= 0 && all_tc && g != 256) {
+        // Overlapped form: the operands of the product that runs first are quantised by the full-size kernel on the
+        // caller's stream; the other product's operands by the small build on the side stream, which shares the SMs
+        // with the small build of the first GEMM (launched by the caller of this function).
+        const int a0 = ov->first == 0 ? 0 : 2, b0 = 2 - a0;             // views (a0, a0 + 1) first, (b0, b0 + 1) hidden
+        const QuantArgs head[2] = {q[a0], q[a0 + 1]}, tail[2] = {q[b0], q[b0 + 1]};
+        if (cuda_status(mx::launch_quantize_tc_group(head, 2, false, stream), "quantiser launch (first product)") != MXFP4_OK) return MXFP4_ERR_CUDA;
+        if (cudaEventRecord(ov->fj->fork, stream) != cudaSuccess || cudaStreamWaitEvent(ov->fj->side, ov->fj->fork, 0) != cudaSuccess) {
+            ov->first = -1;                          // could not fork: the rest of the call stays on the caller's stream
+            return cuda_status(mx::launch_quantize_tc_group(tail, 2, false, stream), "quantiser launch (second product)");
+        }
+        ov->forked = true;
+        return cuda_status(mx::launch_quantize_tc_group(tail, 2, false, ov->fj->side, true), "small quantiser launch (second product)");
+    }
+    if (ov != nullptr) ov->first = -1;
     if (all_tc)                                     // the four views of the call in one launch
-        return cuda_status(mx::launch_quantize_tc_group(q, 4, false, stream), "grouped quantiser launch");
+        return cuda_status(mx::launch_quantize_tc_group(q, 4, false, stream, g != 256 && force_lite()), "grouped quantiser launch");
     for (int i = 0; i < 4; ++i)
         if (cuda_status(mx::launch_quantize(q[i], stream), "quantiser launch") != MXFP4_OK) return MXFP4_ERR_CUDA;
     return MXFP4_OK;
@@ -418,14 +456,38 @@ mxfp4_status linear_backward_impl(const void* dY, const void* X, const void* W, 
     GemmArgs gx, gw;
     if ((st = gemm_prepare(gx, c[0], s[0], c[1], s[1], b, n, m, alpha, dX, n, out_dtype, 0)) != MXFP4_OK) return st;   // dX is never accumulated
     if ((st = gemm_prepare(gw, c[2], s[2], c[3], s[3], m, n, b, alpha, dW, n, out_dtype, accumulate)) != MXFP4_OK) return st;
-    if ((st = quantize_operands_impl(dY, X, W, b, m, n, g, rounding, seed, c, s, stream)) != MXFP4_OK) return st;
-    // Large problems (never the ones the fixed-scratch variant accepts) run the two GEMMs fork / join.
     const int64_t waves_dx = ((b + 255) / 256) * ((n + 255) / 256), waves_dw = ((m + 255) / 256) * ((n + 255) / 256);
+    // Large problems (never the ones the fixed-scratch variant accepts) use a side stream.
     ForkJoin* fj = ws.total > (size_t)MXFP4_STATIC_WORKSPACE_BYTES && waves_dx >= 74 && waves_dw >= 74 ? fork_join() : nullptr;
-    if (fj != nullptr && (cudaEventRecord(fj->fork, stream) != cudaSuccess || cudaStreamWaitEvent(fj->side, fj->fork, 0) != cudaSuccess))
-        fj = nullptr;                                // the side stream was not given anything yet: stay on the caller's stream
-    st = gemm_launch(gx, stream);
-    if (st == MXFP4_OK) st = gemm_launch(gw, fj != nullptr ? fj->side : stream);
+    // Overlapped form (Section 3.2: the transform need not cost GEMM time): quantise the operands of one product, then
+    // run that product's GEMM while the other product's operands are quantised on the same SMs (small builds of both
+    // kernels share an SM: the GEMM keeps the FP4 pipe, the quantiser takes the idle issue slots and ALUs), then the
+    // second GEMM.  The product whose operands are the smaller half goes first, so that more of the quantiser work hides.
+    const int overlap_mode = overlap_setting();
+    Overlap ov{-1, fj};
+    if (fj != nullptr && overlap_mode != 0 && gx.use_pair && gw.use_pair && g != 0 && g != 256) {
+        const int64_t head_dx = b * m + n * m, head_dw = m * b + n * b;       // elements quantised before the first GEMM can start
+        ov.first = overlap_mode == 2 ? 0 : overlap_mode == 3 ? 1 : (head_dx <= head_dw ? 0 : 1);
+    }
+    if ((st = quantize_operands_impl(dY, X, W, b, m, n, g, rounding, seed, c, s, stream, &ov)) != MXFP4_OK) {
+        if (ov.forked && (cudaEventRecord(fj->join, fj->side) != cudaSuccess || cudaStreamWaitEvent(stream, fj->join, 0) != cudaSuccess)) return MXFP4_ERR_CUDA;
+        return st;
+    }
+    if (ov.first >= 0) {
+        GemmArgs& g1 = ov.first == 0 ? gx : gw;
+        GemmArgs& g2 = ov.first == 0 ? gw : gx;
+        g1.lite = true;                              // shares its SMs with the small quantiser running on the side stream
+        st = gemm_launch(g1, stream);
+        const bool joined = cudaEventRecord(fj->join, fj->side) == cudaSuccess && cudaStreamWaitEvent(stream, fj->join, 0) == cudaSuccess;
+        if (!joined) return MXFP4_ERR_CUDA;
+        if (st == MXFP4_OK) st = gemm_launch(g2, stream);
+        fj = nullptr;                                // joined already
+    } else {
+        if (fj != nullptr && (cudaEventRecord(fj->fork, stream) != cudaSuccess || cudaStreamWaitEvent(fj->side, fj->fork, 0) != cudaSuccess))
+            fj = nullptr;                            // the side stream was not given anything yet: stay on the caller's stream
+        st = gemm_launch(gx, stream);
+        if (st == MXFP4_OK) st = gemm_launch(gw, fj != nullptr ? fj->side : stream);
+    }
     // dL/db = 1 dL/dy (problem statement): column sums of dY, after the GEMMs on the caller's stream
     if (st == MXFP4_OK && db != nullptr)
         st = cuda_status(mx::launch_bias_grad(dY, b, m, m, accumulate, db, reinterpret_cast<float*>(base + bias_off), stream), "bias gradient launch");

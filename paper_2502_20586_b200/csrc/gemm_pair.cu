@@ -30,27 +30,39 @@ namespace mx {
 namespace {
 
 constexpr int PM = 256, PN = 256;                           // pair tile
-constexpr int kStagesP = 6;
 constexpr uint32_t kAB = 128 * kGemmBKBytes;                // 16 KB: 128 rows x 128 B, for A and for the B half
 constexpr uint32_t kSfTile = 512;
 constexpr uint32_t kSfaB = 2 * kSfTile;                     // own 128 A rows, 2 tiles (8 K-blocks) per stage
 constexpr uint32_t kSfbB = 2 * 2 * kSfTile;                 // all 256 B rows
 constexpr uint32_t kStageB = 2 * kAB;                       // 32 KB: A rows + B half
-constexpr int kSfSlotsP = kStagesP;                         // scale ring: shared-memory slot i feeds TMEM slot i; same ring
-                                                            // index as the operand stages so ONE commit frees both
 constexpr uint32_t kSfSlotB = kSfaB + kSfbB;                // 3 KB
 constexpr uint32_t kEpiBuf = 2048;                          // epilogue staging: 32 rows x 64 B, two buffers per epilogue warp (4 warps)
 constexpr uint32_t kEpiB = 4 * 2 * kEpiBuf;
 constexpr uint32_t kBarB = 256;
-// The dynamic shared-memory window is at least 256-byte aligned, so rounding its base up to 1024 costs at most 768 bytes.
-constexpr uint32_t kSmemP = kStagesP * kStageB + kSfSlotsP * kSfSlotB + kEpiB + kBarB + 768;
-static_assert(kSmemP <= 232448, "over the 227 KB shared-memory limit");
-constexpr uint32_t kAccColP = 0, kSfColP = 256, kSfSlotColsP = 24;
+constexpr uint32_t kSfSlotColsP = 24;
 constexpr int kGroupMP = 8;                                 // rasterisation: 8 pair-tiles (2048 rows) share B tiles in L2
-// Register hand-over (setmaxnreg) between the three warp groups (kRegsFwdP: the forwarder's group); an increase can only draw on what the CTA holds at
-// launch (threads x registers per thread), which gemm_pair_init checks: an increase that cannot be met waits forever.
-constexpr int kRegsLightP = 56, kRegsFwdP = 64, kRegsEpiP = 232;
 constexpr int kThreadsP = 12 * 32;
+
+// Two builds of the kernel.  FULL owns its SMs: six operand stages (all 227 KB of shared memory), one 512-column TMEM
+// allocation, every register of the SM.  LITE leaves room for a second, independent kernel on the same SM (the
+// tensor-core quantiser's small build, quantize_tc.cu, which quantises the OTHER product's operands meanwhile): four
+// stages, TMEM taken as 256 + 128 columns, 112 registers per thread at launch.
+template <bool LITE>
+struct PairCfg {
+    static constexpr int kStages = LITE ? 4 : 6;
+    static constexpr int kSfSlots = kStages;                // scale ring: shared-memory slot i feeds TMEM slot i; same ring
+                                                            // index as the operand stages so ONE commit frees both
+    // The dynamic shared-memory window is at least 256-byte aligned, so rounding its base up to 1024 costs at most 768 bytes.
+    static constexpr uint32_t kSmem = kStages * kStageB + kSfSlots * kSfSlotB + kEpiB + kBarB + 768;
+    // Register hand-over (setmaxnreg) between the three warp groups (kRegsFwd: the forwarder's group); an increase can only
+    // draw on what the CTA holds at launch (threads x registers per thread), which gemm_pair_init checks: an increase
+    // that cannot be met waits forever.
+    static constexpr int kRegsLight = 56, kRegsFwd = LITE ? 24 : 64, kRegsEpi = 232;
+    static constexpr int kLaunchRegs = LITE ? 104 : 168;    // registers per thread the CTA is given at launch
+    static_assert(kSmem <= 232448, "over the 227 KB shared-memory limit");
+    static_assert(kSfSlots * kSfSlotColsP <= (LITE ? 128 : 256), "scale slots do not fit their TMEM allocation");
+    static_assert(kThreadsP * kLaunchRegs >= 128 * (kRegsLight + kRegsFwd + kRegsEpi), "warp groups ask for more registers than the CTA holds");
+};
 
 struct ParamsP {
     const uint8_t* sfa;
@@ -74,9 +86,10 @@ __device__ __forceinline__ void tile_coords_p(int t, int m_tiles, int n_tiles, i
     nt = r / gm;
 }
 
-__global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(kThreadsP, 1)
-gemm_mxf4_pair_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant__ CUtensorMap tmap_b,
-                      const __grid_constant__ CUtensorMap tmap_c, const ParamsP p) {
+template <bool LITE>
+__device__ __forceinline__ void gemm_pair_body(const CUtensorMap& tmap_a, const CUtensorMap& tmap_b, const CUtensorMap& tmap_c, const ParamsP& p) {
+    using Cfg = PairCfg<LITE>;
+    constexpr int kStagesP = Cfg::kStages, kSfSlotsP = Cfg::kSfSlots;
     extern __shared__ uint8_t smem_raw[];
     uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
     uint8_t* sf_ring = smem + kStagesP * kStageB;
@@ -89,8 +102,8 @@ gemm_mxf4_pair_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_c
     uint64_t* turn = sfl_full + kSfSlotsP;                 // [2] leader: baton between the two MMA issuers
     uint64_t* tmem_full = turn + 2;                         // per CTA: accumulator complete (pair commit)
     uint64_t* tmem_empty = tmem_full + 1;                   // leader: both CTAs drained their accumulators
-    uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(tmem_empty + 1);
-    volatile uint32_t* abort_flag = tmem_slot + 1;
+    uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(tmem_empty + 1);   // [2] base columns of the TMEM allocation(s)
+    volatile uint32_t* abort_flag = tmem_slot + 2;
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const uint32_t rank = cluster_ctarank();                // 0 = leader
@@ -114,14 +127,20 @@ gemm_mxf4_pair_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_c
         if (p.c_tma) prefetch_tensormap(&tmap_c);
     }
     if (warp == 1) {
-        tmem_alloc_pair(tmem_slot, 512);
+        if (LITE) {                                         // accumulator and scale slots as two allocations: 128 columns stay free
+            tmem_alloc_pair(&tmem_slot[0], 256);
+            tmem_alloc_pair(&tmem_slot[1], 128);
+        } else {
+            tmem_alloc_pair(&tmem_slot[0], 512);
+        }
         tmem_relinquish_pair();
     }
     tc_fence_before_sync();
     __syncthreads();
     cluster_sync_all();                                     // both CTAs' barriers exist before anyone signals across
     tc_fence_after_sync();
-    const uint32_t tmem_base = *tmem_slot;
+    const uint32_t tmem_acc = tmem_slot[0];                 // 256 accumulator columns
+    const uint32_t tmem_sf = LITE ? tmem_slot[1] : tmem_slot[0] + 256;   // scale slots of 24 columns
     // Warp group 0 (producer, issuers, scale loader) and warp group 2 (forwarder) need few registers; the epilogue
     // group takes them to hold half an accumulator row and four TMEM loads in flight.
     // Each warp group (four warps) sets its register limit once, at the head of its own branch: all four warps must
@@ -131,7 +150,7 @@ gemm_mxf4_pair_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_c
 
     if (warp < 4) {
     // ============================ warp group 0: producer, two MMA issuers, scale loader (few registers each)
-    reg_dealloc<kRegsLightP>();
+    reg_dealloc<Cfg::kRegsLight>();
     if (warp == 0) {
         // ------------------------------------------------------------------ TMA producer (both CTAs)
         if (lane == 0) {
@@ -166,7 +185,7 @@ gemm_mxf4_pair_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_c
             const uint32_t desc_hi = (uint32_t)(desc0 >> 32);
             const uint32_t a_lo0 = (uint32_t)desc0;
             const bool k_tail = (nkc & 1) != 0;                               // last step holds 128 elements only
-            const uint32_t acc = tmem_base + kAccColP;
+            const uint32_t acc = tmem_acc;
             const uint32_t me = warp == 1 ? 0u : 1u;
             uint32_t s = me % kStagesP, ph = 0, tile_i = 0, n = 0;
             int kt = (int)me;
@@ -176,7 +195,7 @@ gemm_mxf4_pair_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_c
                 if (!(ok = mbar_wait(&full_bar[s], ph, abort_flag))) break;
                 tc_fence_after_sync();
                 const uint32_t a_lo = a_lo0 + s * (kStageB >> 4), b_lo = a_lo + (kAB >> 4);
-                const uint32_t sfa_t = tmem_base + kSfColP + s * kSfSlotColsP, sfb_t = sfa_t + 8;
+                const uint32_t sfa_t = tmem_sf + s * kSfSlotColsP, sfb_t = sfa_t + 8;
                 {   // the step's scales: shared memory -> TMEM of both CTAs, replicated to the four lane quadrants by the copy;
                     // issued while the other thread still issues its MMAs (a different TMEM slot), ordered before this
                     // thread's MMAs by program order
@@ -243,7 +262,7 @@ gemm_mxf4_pair_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_c
     }
     } else if (warp >= 8) {
         // ============================ warp group 2: scale forwarder (warp 8)
-        reg_dealloc<kRegsFwdP>();
+        reg_dealloc<Cfg::kRegsFwd>();
         // The scale copies run in both CTAs on the leader's instruction, so the leader has to know that the peer's tiles
         // have landed too: one thread per CTA passes its ring's completions on to the leader's full barrier.
         bool ok = true;
@@ -257,7 +276,7 @@ gemm_mxf4_pair_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_c
         if (!ok && lane == 0) *abort_flag = 1;
     } else {
         // ------------------------------------------------------------------ epilogue (both CTAs, own 128 rows)
-        reg_alloc<kRegsEpiP>();                                   // warp group 1 takes the registers the others gave up
+        reg_alloc<Cfg::kRegsEpi>();                                  // warp group 1 takes the registers the others gave up
         // TMEM -> registers -> (alpha, convert) -> shared memory -> TMA store.  Each warp owns the 32 accumulator
         // lanes of its quadrant and two 2 KB staging buffers (32 rows x 64 bytes, 64-byte swizzle, so the row-per-lane
         // writes are conflict-free); the accumulator is handed back as soon as its last column is in registers.
@@ -307,7 +326,7 @@ gemm_mxf4_pair_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_c
                     uint32_t r[4][32];
 #pragma unroll
                     for (int c = 0; c < 4; ++c)
-                        tmem_ld_32x32b_x32(tmem_base + kAccColP + ((uint32_t)(q * 32) << 16) + (4 * hb + c) * 32, r[c]);
+                        tmem_ld_32x32b_x32(tmem_acc + ((uint32_t)(q * 32) << 16) + (4 * hb + c) * 32, r[c]);
                     tmem_ld_wait();
                     if (hb == 1) {                              // the accumulator is in registers: hand it back before converting
                         tc_fence_before_sync();
@@ -336,7 +355,7 @@ gemm_mxf4_pair_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_c
 #pragma unroll 1
             for (int c = 0; c < n_chunks; ++c) {
                 uint32_t r[32];
-                tmem_ld_32x32b_x32(tmem_base + kAccColP + ((uint32_t)(q * 32) << 16) + c * 32, r);
+                tmem_ld_32x32b_x32(tmem_acc + ((uint32_t)(q * 32) << 16) + c * 32, r);
                 tmem_ld_wait();
                 if (c == n_chunks - 1) {                        // accumulator drained: the next tile's MMAs may start
                     tc_fence_before_sync();
@@ -410,22 +429,51 @@ gemm_mxf4_pair_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_c
     cluster_sync_all();                                     // neither CTA leaves while the other may still signal it
     if (warp == 1) {
         tc_fence_after_sync();
-        tmem_dealloc_pair(tmem_base, 512);
+        if (LITE) {
+            tmem_dealloc_pair(tmem_slot[1], 128);
+            tmem_dealloc_pair(tmem_slot[0], 256);
+        } else {
+            tmem_dealloc_pair(tmem_slot[0], 512);
+        }
     }
+}
+
+__global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(kThreadsP, 1)
+gemm_mxf4_pair_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant__ CUtensorMap tmap_b,
+                      const __grid_constant__ CUtensorMap tmap_c, const ParamsP p) {
+    gemm_pair_body<false>(tmap_a, tmap_b, tmap_c, p);
+}
+
+// The small-footprint build (see PairCfg): same roles, same arithmetic, same accumulation order.
+__global__ void __cluster_dims__(2, 1, 1) __maxnreg__(PairCfg<true>::kLaunchRegs)
+gemm_mxf4_pair_lite_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant__ CUtensorMap tmap_b,
+                           const __grid_constant__ CUtensorMap tmap_c, const ParamsP p) {
+    gemm_pair_body<true>(tmap_a, tmap_b, tmap_c, p);
 }
 
 }  // namespace
 
 cudaError_t fetch_gemm_pair_status(unsigned int* word) { return device_status_fetch(word); }
 
-cudaError_t gemm_pair_init() {
-    cudaError_t e = cudaFuncSetAttribute(gemm_mxf4_pair_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kSmemP);
+template <bool LITE, typename K>
+static cudaError_t pair_kernel_init(K kernel) {
+    using Cfg = PairCfg<LITE>;
+    cudaError_t e = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)Cfg::kSmem);
+    if (e != cudaSuccess) return e;
+    // All of the SM's configurable memory as shared memory: two kernels can only share an SM under one carve-out, and
+    // the small builds of GEMM and quantiser together need nearly all of it.
+    e = cudaFuncSetAttribute(kernel, cudaFuncAttributePreferredSharedMemoryCarveout, (int)cudaSharedmemCarveoutMaxShared);
     if (e != cudaSuccess) return e;
     cudaFuncAttributes fa;
-    e = cudaFuncGetAttributes(&fa, gemm_mxf4_pair_kernel);
+    e = cudaFuncGetAttributes(&fa, kernel);
     if (e != cudaSuccess) return e;
-    if (fa.numRegs * kThreadsP < 128 * (kRegsLightP + kRegsFwdP + kRegsEpiP)) return cudaErrorLaunchOutOfResources;
+    if (fa.numRegs * kThreadsP < 128 * (Cfg::kRegsLight + Cfg::kRegsFwd + Cfg::kRegsEpi)) return cudaErrorLaunchOutOfResources;
     return cudaSuccess;
+}
+
+cudaError_t gemm_pair_init() {
+    const cudaError_t e = pair_kernel_init<false>(gemm_mxf4_pair_kernel);
+    return e != cudaSuccess ? e : pair_kernel_init<true>(gemm_mxf4_pair_lite_kernel);
 }
 
 cudaError_t launch_gemm_pair(const GemmArgs& a, cudaStream_t stream) {
@@ -445,12 +493,13 @@ cudaError_t launch_gemm_pair(const GemmArgs& a, cudaStream_t stream) {
     p.c_tma = a.has_tmap_c ? 1 : 0;
     p.accumulate = a.accumulate;
     cudaLaunchConfig_t cfg = {};
-    cfg.gridDim = dim3(2 * pairs); cfg.blockDim = dim3(kThreadsP); cfg.dynamicSmemBytes = kSmemP; cfg.stream = stream;
+    cfg.gridDim = dim3(2 * pairs); cfg.blockDim = dim3(kThreadsP); cfg.stream = stream;
+    cfg.dynamicSmemBytes = a.lite ? PairCfg<true>::kSmem : PairCfg<false>::kSmem;
     cudaLaunchAttribute attr[1];
     attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
     attr[0].val.programmaticStreamSerializationAllowed = 1;
     cfg.attrs = attr; cfg.numAttrs = 1;
-    return cudaLaunchKernelEx(&cfg, gemm_mxf4_pair_kernel, a.tmap_a, a.tmap_b_half, a.tmap_c, p);
+    return cudaLaunchKernelEx(&cfg, a.lite ? gemm_mxf4_pair_lite_kernel : gemm_mxf4_pair_kernel, a.tmap_a, a.tmap_b_half, a.tmap_c, p);
 }
 
 }  // namespace mx

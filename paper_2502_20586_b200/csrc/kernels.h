@@ -29,7 +29,8 @@ cudaError_t quant_tc_init();
 cudaError_t launch_quantize_tc(const QuantArgs& a, bool dump_y, cudaStream_t stream);
 // Up to kQuantMaxViews eligible views sharing g, seed, rounding and scale layout, in ONE launch.
 constexpr int kQuantMaxViews = 4;
-cudaError_t launch_quantize_tc_group(const QuantArgs* a, int n, bool dump_y, cudaStream_t stream);
+// lite: the small-footprint build (g <= 128) that can share an SM with the small build of the pair GEMM.
+cudaError_t launch_quantize_tc_group(const QuantArgs* a, int n, bool dump_y, cudaStream_t stream, bool lite = false);
 
 cudaError_t launch_quantize(const QuantArgs& a, cudaStream_t stream);
 cudaError_t launch_rht_dump(const QuantArgs& a, cudaStream_t stream);
@@ -41,6 +42,7 @@ struct GemmArgs {
     CUtensorMap tmap_c;   // output [M, N] (leading dimension ldc): box 64 bytes x 32 rows, 64-byte swizzle (pair kernel's stores)
     bool has_tmap_c;      // false when C cannot be described by a tensor map: the kernel then stores directly
     bool use_pair;        // run the CTA-pair kernel (gemm_pair.cu)
+    bool lite = false;    // pair kernel only: the small-footprint build that leaves room on the SM for a co-resident quantiser
     const uint8_t* sfa;   // native scale layout
     const uint8_t* sfb;
     int64_t M, N, K;

@@ -35,19 +35,31 @@ namespace mx {
 namespace {
 
 constexpr int kTile = 128;                          // output rows per tile and reduce-dim elements per tile
-constexpr int kStagesQ = 4;
 constexpr uint32_t kBoxBytes = 64 * 2 * 128;        // one TMA box: 64 bf16 columns x 128 rows = 16 KB
 constexpr uint32_t kTileBytes = 2 * kBoxBytes;      // 32 KB
 constexpr uint32_t kTBytes = 2 * kBoxBytes;         // transform matrix, 128 x 128 bf16
-constexpr uint32_t kSmemQ = kStagesQ * kTileBytes + 2 * kTBytes + 1024 + 256;   // two transform matrices for g = 256
-constexpr int kAccBufs = 4;                         // 4 x 128 TMEM columns
-constexpr int kEpiGroups = 4;                       // epilogue warp groups (one warp per TMEM lane quadrant), on alternate tiles
-constexpr int kEpiWarps = 4 * kEpiGroups;
-// Register hand-over (setmaxnreg): warp group 0 shrinks to kRegsLight, the epilogue groups grow to kRegsEpi.  The
-// increase can only draw on what the CTA itself holds, i.e. threads x registers-per-thread at launch: the init
-// routine checks that budget against the compiled kernel, because an increase that cannot be met waits forever.
-constexpr int kRegsLight = 40, kRegsEpi = 104;
-constexpr int kThreadsQ = (4 + kEpiWarps) * 32;    // warp group 0: producer, MMA issuer, two idle warps; then the epilogue warp groups
+
+// Two builds of the kernel.  FULL owns its SM: a 4-stage ring, four TMEM accumulators, four epilogue warp groups on
+// alternate tiles.  LITE is sized to run beside the small build of the pair GEMM (gemm_pair.cu) on the same SM, so that
+// the operands of one product are quantised while the other product's GEMM keeps the FP4 pipe busy: one 32 KB stage,
+// one accumulator (128 TMEM columns), two epilogue warp groups that share every tile (two MX blocks of each row per
+// group), 64 registers per thread at launch.  g <= 128 only.  Codes and scales are the same bytes in both builds.
+template <bool LITE>
+struct QCfg {
+    static constexpr int kStages = LITE ? 1 : 4;
+    static constexpr int kAccBufs = LITE ? 1 : 4;                        // x 128 TMEM columns
+    static constexpr int kTmemCols = LITE ? 128 : 512;
+    static constexpr int kEpiGroups = LITE ? 2 : 4;                      // epilogue warp groups (one warp per TMEM lane quadrant)
+    static constexpr int kEpiWarps = 4 * kEpiGroups;
+    static constexpr uint32_t kSmem = kStages * kTileBytes + (LITE ? 1 : 2) * kTBytes + 1024 + 256;   // FULL: two transform matrices for g = 256
+    // Register hand-over (setmaxnreg): warp group 0 shrinks to kRegsLight, the epilogue groups grow to kRegsEpi.  The
+    // increase can only draw on what the CTA itself holds, i.e. threads x registers-per-thread at launch: the init
+    // routine checks that budget against the compiled kernel, because an increase that cannot be met waits forever.
+    static constexpr int kRegsLight = LITE ? 32 : 40, kRegsEpi = LITE ? 80 : 104;
+    static constexpr int kThreads = (4 + kEpiWarps) * 32;                // warp group 0: producer, MMA issuer, two idle warps; then the epilogue warp groups
+    static constexpr int kLaunchRegs = LITE ? 64 : 96;
+    static_assert(kThreads * kLaunchRegs >= 128 * kRegsLight + (kThreads - 128) * kRegsEpi, "warp groups ask for more registers than the CTA holds");
+};
 
 struct QView {                 // one operand view: output operand [R, K] read from x [rows, cols]
     int64_t R, K;
@@ -127,13 +139,15 @@ __device__ __forceinline__ void view_draws32(const PhiloxKeys& ks, uint32_t stre
 }
 
 // KW = 128-wide k-tiles per entry of the tile list: 1, or 2 for g = 256 (a tile then spans one 256-chunk).
-template <int MODE, int KW>
-__global__ void __launch_bounds__(kThreadsQ, 1)
-quantize_tc_kernel(const __grid_constant__ QMaps maps, const __grid_constant__ QParams p) {
+template <int MODE, int KW, bool LITE>
+__device__ __forceinline__ void quantize_tc_body(const QMaps& maps, const QParams& p) {
+    using Cfg = QCfg<LITE>;
+    constexpr int kStagesQ = Cfg::kStages, kAccBufs = Cfg::kAccBufs, kEpiGroups = Cfg::kEpiGroups, kThreadsQ = Cfg::kThreads;
+    static_assert(!(LITE && KW == 2), "the small build serves g <= 128");
     extern __shared__ uint8_t smem_raw[];
     uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
     uint8_t* smem_t = smem + kStagesQ * kTileBytes;
-    uint64_t* bars = reinterpret_cast<uint64_t*>(smem_t + 2 * kTBytes);
+    uint64_t* bars = reinterpret_cast<uint64_t*>(smem_t + (LITE ? 1 : 2) * kTBytes);
     uint64_t* full_bar = bars;                          // [kStagesQ]  TMA -> MMA
     uint64_t* empty_bar = bars + kStagesQ;              // [kStagesQ]  MMA -> TMA
     uint64_t* acc_full = bars + 2 * kStagesQ;           // [kAccBufs]  MMA -> epilogue
@@ -147,13 +161,13 @@ quantize_tc_kernel(const __grid_constant__ QMaps maps, const __grid_constant__ Q
 
     if (threadIdx.x == 0) {
         for (int s = 0; s < kStagesQ; ++s) { mbar_init(&full_bar[s], 1); mbar_init(&empty_bar[s], 1); }
-        for (int b = 0; b < kAccBufs; ++b) { mbar_init(&acc_full[b], 1); mbar_init(&acc_empty[b], KW == 2 ? 8 : 4); }
+        for (int b = 0; b < kAccBufs; ++b) { mbar_init(&acc_full[b], 1); mbar_init(&acc_empty[b], (KW == 2 || LITE) ? 8 : 4); }
         *abort_flag = 0;
         mbar_fence_init();
         for (int v = 0; v < p.n_views; ++v) prefetch_tensormap(&maps.x[v]);
     }
     if (warp == 1) {
-        tmem_alloc(tmem_slot, 512);
+        tmem_alloc(tmem_slot, Cfg::kTmemCols);
         tmem_relinquish();
     }
     {
@@ -197,7 +211,7 @@ quantize_tc_kernel(const __grid_constant__ QMaps maps, const __grid_constant__ Q
 
     if (warp < 4) {
     // ============================ warp group 0: producer, MMA issuer, two idle warps; it gives registers to the others
-    reg_dealloc<kRegsLight>();
+    reg_dealloc<Cfg::kRegsLight>();
     if (warp == 0) {
         // ------------------------------------------------------------------ TMA producer
         if (lane == 0) {
@@ -263,7 +277,7 @@ quantize_tc_kernel(const __grid_constant__ QMaps maps, const __grid_constant__ Q
     }
     } else {
         // ------------------------------------------------------------------ epilogue (warp groups 1..4)
-        reg_alloc<kRegsEpi>();
+        reg_alloc<Cfg::kRegsEpi>();
         // Four groups of four warps take alternate tiles; inside a group a warp owns one TMEM lane quadrant, i.e. a
         // thread owns one output row of the tile: four MX blocks, 64 bytes of codes, 4 scale bytes.  The SR draws of a
         // block are computed while the block before it is rounded (for a tile's first block: at the end of the tile
@@ -272,7 +286,11 @@ quantize_tc_kernel(const __grid_constant__ QMaps maps, const __grid_constant__ Q
         const int q = warp & 3;                      // TMEM lane quadrant this warp may read
         const int grp = e >> 2;
         const float cg = p.custom_t != nullptr ? 1.0f : p.g == 32 ? 0.17677669529663687f : p.g == 128 ? 0.08838834764831845f : 1.0f;
-        const uint32_t stride = (uint32_t)kEpiGroups * gridDim.x;
+        // FULL: the groups take alternate tiles.  LITE: both groups take every tile of the CTA, group 0 the row's MX
+        // blocks 0 and 1, group 1 blocks 2 and 3.
+        const uint32_t stride = (LITE ? 1u : (uint32_t)kEpiGroups) * gridDim.x;
+        constexpr int kBlocksPerThread = LITE ? 2 : 4;
+        const int jb = LITE ? 2 * grp : 0;                          // first MX block of the row this thread handles
         const uint32_t lane_row = (uint32_t)(q * 32 + lane);
         bool ok = true;
 
@@ -280,11 +298,11 @@ quantize_tc_kernel(const __grid_constant__ QMaps maps, const __grid_constant__ Q
             return (uint64_t)(pos.rt * (uint32_t)kTile + lane_row) * (uint64_t)p.view[pos.v].K + (uint64_t)(pos.kt * (uint32_t)(kTile * KW));
         };
 
-        uint32_t it = (uint32_t)grp;
+        uint32_t it = LITE ? 0u : (uint32_t)grp;
         uint32_t t = blockIdx.x + it * gridDim.x;
         TilePos pos = locate_tile(p, t < num_tiles ? t : 0u);
         uint32_t rw[8];
-        if (mode_draws(MODE)) view_draws32<kFold>(p.keys, p.view[pos.v].stream_tag, &p.view[pos.v].pv, first_elem(pos), rw);
+        if (mode_draws(MODE)) view_draws32<kFold>(p.keys, p.view[pos.v].stream_tag, &p.view[pos.v].pv, first_elem(pos) + 32u * jb, rw);
         if (KW == 2) {
             // g = 256: a tile is one 256-chunk of 128 rows; its two k-tiles went through T_0 and T_1 into the accumulator
             // pair (b0, b0 + 1): u = A_lo T_0, v = A_hi T_1.  The transformed values are y[0..127] = u + v and
@@ -365,7 +383,7 @@ quantize_tc_kernel(const __grid_constant__ QMaps maps, const __grid_constant__ Q
                 if (MODE != kModeDump && live) *reinterpret_cast<uint32_t*>(scale_dst) = sb_all;
             }
         } else
-        for (; t < num_tiles; t += stride, it += kEpiGroups) {
+        for (; t < num_tiles; t += stride, it += (LITE ? 1 : kEpiGroups)) {
             const int b = it % kAccBufs;
             const QView& vw = p.view[pos.v];
             const uint32_t rt = pos.rt, kt = pos.kt;
@@ -392,19 +410,20 @@ quantize_tc_kernel(const __grid_constant__ QMaps maps, const __grid_constant__ Q
             const uint32_t taddr = tmem_base + ((uint32_t)(q * 32) << 16) + b * kTile;
             uint32_t sb_all = 0;
 #pragma unroll
-            for (int j = 0; j < 4; ++j) {
+            for (int jj = 0; jj < kBlocksPerThread; ++jj) {
+                const int j = jb + jj;                          // MX block of the row
                 uint32_t raw[32], nx[8], packed[4], sb = 0;
                 float y[32];
                 tmem_ld_32x32b_x32(taddr + 32 * j, raw);
                 tmem_ld_wait();
-                if (j == 3) {                                   // the accumulator is free once it has been read
+                if (jj == kBlocksPerThread - 1) {               // the accumulator is free once it has been read
                     tc_fence_before_sync();
                     __syncwarp();
                     if (lane == 0) mbar_arrive(&acc_empty[b]);
                 }
                 if (mode_draws(MODE)) {
-                    if (j < 3) view_draws32<kFold>(p.keys, tag_cur, pv_cur, i_cur + 32 * (j + 1), nx);
-                    else view_draws32<kFold>(p.keys, tag_next, pv_next, i_next, nx);
+                    if (jj < kBlocksPerThread - 1) view_draws32<kFold>(p.keys, tag_cur, pv_cur, i_cur + 32 * (j + 1), nx);
+                    else view_draws32<kFold>(p.keys, tag_next, pv_next, i_next + 32u * jb, nx);
                 }
 #pragma unroll
                 for (int i = 0; i < 32; ++i) y[i] = __uint_as_float(raw[i]);
@@ -421,15 +440,17 @@ quantize_tc_kernel(const __grid_constant__ QMaps maps, const __grid_constant__ Q
                 } else {
                     quantize_block32_rw<mode_rounding(MODE, KW)>(y, rw, packed, sb, p.pipe);
                     if (live) *reinterpret_cast<uint4*>(code_dst + 16 * j) = make_uint4(packed[0], packed[1], packed[2], packed[3]);
-                    sb_all |= sb << (8 * j);
+                    sb_all |= sb << (8 * jj);
                 }
                 if (mode_draws(MODE)) {
 #pragma unroll
                     for (int i = 0; i < 8; ++i) rw[i] = nx[i];
                 }
             }
-            if (MODE != kModeDump && live)
-                *reinterpret_cast<uint32_t*>(scale_dst) = sb_all;       // four consecutive bytes in either scale layout
+            if (MODE != kModeDump && live) {
+                if (LITE) *reinterpret_cast<uint16_t*>(scale_dst + jb) = (uint16_t)sb_all;   // this group's two of the row's four scale bytes
+                else *reinterpret_cast<uint32_t*>(scale_dst) = sb_all;                     // four consecutive bytes in either scale layout
+            }
         }
         if (!ok && lane == 0) *abort_flag = 1;
     }
@@ -442,8 +463,21 @@ quantize_tc_kernel(const __grid_constant__ QMaps maps, const __grid_constant__ Q
     }
     if (warp == 1) {
         tc_fence_after_sync();
-        tmem_dealloc(tmem_base, 512);
+        tmem_dealloc(tmem_base, Cfg::kTmemCols);
     }
+}
+
+template <int MODE, int KW>
+__global__ void __launch_bounds__(QCfg<false>::kThreads, 1)
+quantize_tc_kernel(const __grid_constant__ QMaps maps, const __grid_constant__ QParams p) {
+    quantize_tc_body<MODE, KW, false>(maps, p);
+}
+
+// The small-footprint build (see QCfg), g <= 128.
+template <int MODE>
+__global__ void __maxnreg__(QCfg<true>::kLaunchRegs)
+quantize_tc_lite_kernel(const __grid_constant__ QMaps maps, const __grid_constant__ QParams p) {
+    quantize_tc_body<MODE, 1, true>(maps, p);
 }
 
 }  // namespace
@@ -459,26 +493,44 @@ bool quant_tc_eligible(const QuantArgs& a) {
 
 cudaError_t fetch_quant_tc_status(unsigned int* word) { return device_status_fetch(word); }
 
+template <bool LITE>
+static cudaError_t quant_kernel_init(const void* k) {
+    using Cfg = QCfg<LITE>;
+    cudaError_t e = cudaFuncSetAttribute(k, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)Cfg::kSmem);
+    if (e != cudaSuccess) return e;
+    // all of the SM's configurable memory as shared memory (see gemm_pair.cu: kernels share an SM only under one carve-out)
+    e = cudaFuncSetAttribute(k, cudaFuncAttributePreferredSharedMemoryCarveout, (int)cudaSharedmemCarveoutMaxShared);
+    if (e != cudaSuccess) return e;
+    cudaFuncAttributes fa;
+    e = cudaFuncGetAttributes(&fa, k);
+    if (e != cudaSuccess) return e;
+    // registers the CTA holds at launch must cover the limits the warp groups set for themselves
+    if (fa.numRegs * Cfg::kThreads < 128 * Cfg::kRegsLight + (Cfg::kThreads - 128) * Cfg::kRegsEpi) return cudaErrorLaunchOutOfResources;
+    return cudaSuccess;
+}
+
 cudaError_t quant_tc_init() {
     const void* kernels[8] = {(const void*)quantize_tc_kernel<kModeSR, 1>, (const void*)quantize_tc_kernel<kModeRN, 1>,
                               (const void*)quantize_tc_kernel<kModeDump, 1>, (const void*)quantize_tc_kernel<kModeSR16, 1>,
                               (const void*)quantize_tc_kernel<kModeSR, 2>, (const void*)quantize_tc_kernel<kModeRN, 2>,
                               (const void*)quantize_tc_kernel<kModeDump, 2>, (const void*)quantize_tc_kernel<kModeSR16, 2>};
     for (const void* k : kernels) {
-        cudaError_t e = cudaFuncSetAttribute(k, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kSmemQ);
+        const cudaError_t e = quant_kernel_init<false>(k);
         if (e != cudaSuccess) return e;
-        cudaFuncAttributes fa;
-        e = cudaFuncGetAttributes(&fa, k);
+    }
+    const void* lite[3] = {(const void*)quantize_tc_lite_kernel<kModeSR>, (const void*)quantize_tc_lite_kernel<kModeRN>,
+                           (const void*)quantize_tc_lite_kernel<kModeSR16>};
+    for (const void* k : lite) {
+        const cudaError_t e = quant_kernel_init<true>(k);
         if (e != cudaSuccess) return e;
-        // registers the CTA holds at launch must cover the limits the warp groups set for themselves
-        if (fa.numRegs * kThreadsQ < 128 * kRegsLight + (kThreadsQ - 128) * kRegsEpi) return cudaErrorLaunchOutOfResources;
     }
     return cudaSuccess;
 }
 
 // Quantise n (1..kQuantMaxViews) eligible operand views that share g, seed, rounding and scale layout in one launch.
-cudaError_t launch_quantize_tc_group(const QuantArgs* a, int n, bool dump_y, cudaStream_t stream) {
+cudaError_t launch_quantize_tc_group(const QuantArgs* a, int n, bool dump_y, cudaStream_t stream, bool lite) {
     if (n < 1 || n > kQuantMaxViews) return cudaErrorInvalidValue;
+    if (lite && (dump_y || a[0].g == 256 || a[0].custom_t != nullptr)) return cudaErrorInvalidValue;   // the small build: RHT with g <= 128, quantising
     QParams p;
     QMaps maps;
     uint32_t tiles = 0;
@@ -517,21 +569,25 @@ cudaError_t launch_quantize_tc_group(const QuantArgs* a, int n, bool dump_y, cud
     e = cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
     if (e != cudaSuccess) return e;
     const unsigned grid = tiles < (uint32_t)sms ? tiles : (unsigned)sms;
-    for (int v = 0; v < kQuantMaxViews; ++v) {              // the two epilogue groups step through the list by 2 * grid
+    for (int v = 0; v < kQuantMaxViews; ++v) {
         QView& w = p.view[v];
         w.minor_count = w.reduce_dim == 1 ? w.k_tiles : w.r_tiles;
-        const uint32_t step = (p.g == 256 ? 2u : (uint32_t)kEpiGroups) * grid;   // g = 256: the groups work in pairs
+        // tiles between two visits of an epilogue group: the groups take alternate tiles (g = 256: in pairs; small build: every tile)
+        const uint32_t step = (lite ? 1u : p.g == 256 ? 2u : (uint32_t)QCfg<false>::kEpiGroups) * grid;
         w.d_major = step / w.minor_count;
         w.d_minor = step % w.minor_count;
     }
     const bool wide = p.g == 256;
     void (*kernel)(QMaps, QParams);
-    if (dump_y) kernel = wide ? quantize_tc_kernel<kModeDump, 2> : quantize_tc_kernel<kModeDump, 1>;
+    if (lite) kernel = a[0].rounding == 0 ? quantize_tc_lite_kernel<kModeSR> : a[0].rounding == 2 ? quantize_tc_lite_kernel<kModeSR16> : quantize_tc_lite_kernel<kModeRN>;
+    else if (dump_y) kernel = wide ? quantize_tc_kernel<kModeDump, 2> : quantize_tc_kernel<kModeDump, 1>;
     else if (a[0].rounding == 0) kernel = wide ? quantize_tc_kernel<kModeSR, 2> : quantize_tc_kernel<kModeSR, 1>;
     else if (a[0].rounding == 2) kernel = wide ? quantize_tc_kernel<kModeSR16, 2> : quantize_tc_kernel<kModeSR16, 1>;
     else kernel = wide ? quantize_tc_kernel<kModeRN, 2> : quantize_tc_kernel<kModeRN, 1>;
     cudaLaunchConfig_t cfg = {};
-    cfg.gridDim = dim3(grid); cfg.blockDim = dim3(kThreadsQ); cfg.dynamicSmemBytes = kSmemQ; cfg.stream = stream;
+    cfg.gridDim = dim3(grid); cfg.stream = stream;
+    cfg.blockDim = dim3(lite ? QCfg<true>::kThreads : QCfg<false>::kThreads);
+    cfg.dynamicSmemBytes = lite ? QCfg<true>::kSmem : QCfg<false>::kSmem;
     cudaLaunchAttribute attr[1];
     attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
     attr[0].val.programmaticStreamSerializationAllowed = 1;
@@ -540,7 +596,7 @@ cudaError_t launch_quantize_tc_group(const QuantArgs* a, int n, bool dump_y, cud
 }
 
 cudaError_t launch_quantize_tc(const QuantArgs& a, bool dump_y, cudaStream_t stream) {
-    return launch_quantize_tc_group(&a, 1, dump_y, stream);
+    return launch_quantize_tc_group(&a, 1, dump_y, stream, false);
 }
 
 }  // namespace mx
