@@ -124,6 +124,12 @@ bool force_lite() {
     return e != nullptr && e[0] == '1';
 }
 
+// MXFP4_DUAL_DY=0: quantise the two views of dY as separate tile lists (two reads of dY) instead of one read for both.
+bool dual_setting() {
+    const char* e = getenv("MXFP4_DUAL_DY");
+    return !(e != nullptr && e[0] == '0');
+}
+
 int overlap_setting() {
     const char* e = getenv("MXFP4_OVERLAP");
     if (e == nullptr || e[0] == '\0') return 0;
@@ -407,6 +413,12 @@ mxfp4_status quantize_operands_impl(const void* dY, const void* X, const void* W
         return cuda_status(mx::launch_quantize_tc_group(tail, 2, false, ov->fj->side, true), "small quantiser launch (second product)");
     }
     if (ov != nullptr) ov->first = -1;
+    if (all_tc && g != 256 && !force_lite() && dual_setting()) {
+        // dL/dy feeds lines 3 and 5: its two views come from ONE read of it; W^T and X^T in a second launch
+        const QuantArgs dy[2] = {q[0], q[2]}, wx[2] = {q[1], q[3]};
+        if (cuda_status(mx::launch_quantize_tc_group(dy, 2, false, stream, false, true), "quantiser launch (both views of dY)") != MXFP4_OK) return MXFP4_ERR_CUDA;
+        return cuda_status(mx::launch_quantize_tc_group(wx, 2, false, stream), "quantiser launch (W, X)");
+    }
     if (all_tc)                                     // the four views of the call in one launch
         return cuda_status(mx::launch_quantize_tc_group(q, 4, false, stream, g != 256 && force_lite()), "grouped quantiser launch");
     for (int i = 0; i < 4; ++i)

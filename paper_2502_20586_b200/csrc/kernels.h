@@ -30,7 +30,8 @@ cudaError_t launch_quantize_tc(const QuantArgs& a, bool dump_y, cudaStream_t str
 // Up to kQuantMaxViews eligible views sharing g, seed, rounding and scale layout, in ONE launch.
 constexpr int kQuantMaxViews = 4;
 // lite: the small-footprint build (g <= 128) that can share an SM with the small build of the pair GEMM.
-cudaError_t launch_quantize_tc_group(const QuantArgs* a, int n, bool dump_y, cudaStream_t stream, bool lite = false);
+// dual: n = 2, a[0] / a[1] = the row-wise and the transposed view of ONE tensor (both extents multiples of 128): every tile of it is read once.
+cudaError_t launch_quantize_tc_group(const QuantArgs* a, int n, bool dump_y, cudaStream_t stream, bool lite = false, bool dual = false);
 
 cudaError_t launch_quantize(const QuantArgs& a, cudaStream_t stream);
 cudaError_t launch_rht_dump(const QuantArgs& a, cudaStream_t stream);

@@ -125,6 +125,19 @@ __device__ __forceinline__ TilePos advance_tile(const QParams& p, const TilePos&
     return pos;
 }
 
+// DUAL launches: view 0 (reduce along x columns) and view 1 (reduce along x rows) are the two views of ONE tensor x
+// (dY of Algorithm 3, lines 3 and 5).  A unit is one 128 x 128 tile of x, loaded once; it yields two logical tiles,
+// 2 u (view 0: rows = x rows) and 2 u + 1 (view 1: rows = x columns).  Units run along x columns first.
+__device__ __forceinline__ TilePos locate_dual(const QParams& p, uint32_t t) {
+    const uint32_t u = t >> 1, xc_tiles = p.view[0].k_tiles;
+    const uint32_t xr = u / xc_tiles, xc = u - xr * xc_tiles;
+    TilePos pos;
+    pos.v = (int)(t & 1u);
+    pos.local = u;
+    if (pos.v == 0) { pos.rt = xr; pos.kt = xc; } else { pos.rt = xc; pos.kt = xr; }
+    return pos;
+}
+
 enum { kModeSR = 0, kModeRN = 1, kModeDump = 2, kModeSR16 = 3 };
 constexpr bool mode_draws(int mode) { return mode == kModeSR || mode == kModeSR16; }
 // template argument of quantize_block32_rw; the g = 256 kernel (kw = 2) rounds SR through the convert instruction (same codes, fewer registers)
@@ -139,9 +152,10 @@ __device__ __forceinline__ void view_draws32(const PhiloxKeys& ks, uint32_t stre
 }
 
 // KW = 128-wide k-tiles per entry of the tile list: 1, or 2 for g = 256 (a tile then spans one 256-chunk).
-template <int MODE, int KW, bool LITE>
+template <int MODE, int KW, bool LITE, bool DUAL>
 __device__ __forceinline__ void quantize_tc_body(const QMaps& maps, const QParams& p) {
     using Cfg = QCfg<LITE>;
+    static_assert(!DUAL || (KW == 1 && !LITE), "one load for two views: g <= 128, full-size build");
     constexpr int kStagesQ = Cfg::kStages, kAccBufs = Cfg::kAccBufs, kEpiGroups = Cfg::kEpiGroups, kThreadsQ = Cfg::kThreads;
     static_assert(!(LITE && KW == 2), "the small build serves g <= 128");
     extern __shared__ uint8_t smem_raw[];
@@ -217,8 +231,9 @@ __device__ __forceinline__ void quantize_tc_body(const QMaps& maps, const QParam
         if (lane == 0) {
             uint32_t it = 0;
             bool ok = true;
-            for (uint32_t t = blockIdx.x; t < num_tiles && ok; t += gridDim.x) {
-                const TilePos pos = locate_tile(p, t);
+            // DUAL: one load per unit (two logical tiles), in the coordinates of its row-wise view
+            for (uint32_t t = DUAL ? 2u * blockIdx.x : blockIdx.x; t < num_tiles && ok; t += (DUAL ? 2u : 1u) * gridDim.x) {
+                const TilePos pos = DUAL ? locate_dual(p, t) : locate_tile(p, t);
                 // x coordinates: (column, row).  reduce_dim 1: output rows = x rows, k = x columns; else swapped.
                 const bool rowwise = p.view[pos.v].reduce_dim == 1;
 #pragma unroll
@@ -244,30 +259,49 @@ __device__ __forceinline__ void quantize_tc_body(const QMaps& maps, const QParam
             const uint32_t t_addr = smem_u32(smem_t);
             uint32_t it = 0;
             bool ok = true;
+            auto transform = [&](uint32_t a_addr, bool rowwise, int h, int b) {      // 8 MMAs: stage -> accumulator b
+                const uint32_t idesc = idesc_k | ((rowwise ? 0u : 1u) << 15);
+#pragma unroll
+                for (int ks = 0; ks < 8; ++ks) {                           // K = 16 per MMA
+                    uint64_t adesc;
+                    if (rowwise)            // K-major: box ks/4, 32 bytes of K per step inside the 128-byte swizzle atom
+                        adesc = make_smem_desc(a_addr + (ks >> 2) * kBoxBytes + (ks & 3) * 32, 16, 1024, 2);
+                    else                    // MN-major: 16 k-rows of 128 B per step; the second 64 output rows sit one box further
+                        adesc = make_smem_desc(a_addr + ks * 2048, kBoxBytes, 1024, 2);
+                    const uint64_t bdesc = make_smem_desc(t_addr + h * kTBytes + (ks >> 2) * kBoxBytes + (ks & 3) * 32, 16, 1024, 2);
+                    tc_mma_f16(tmem_base + b * kTile, adesc, bdesc, idesc, ks != 0 ? 1u : 0u);
+                }
+            };
+            if (DUAL) {
+                // per unit: the stage is the K-major operand of view 0's transform and the MN-major operand of view 1's
+                uint32_t is = 0;                                             // stage counter (units)
+                for (uint32_t u = blockIdx.x; 2u * u < num_tiles && ok; u += gridDim.x, ++is) {
+                    const int s = is % kStagesQ;
+                    if (!(ok = mbar_wait(&full_bar[s], (is / kStagesQ) & 1, abort_flag))) break;
+                    const uint32_t a_addr = smem_u32(smem + s * kTileBytes);
+                    for (int h = 0; h < 2 && ok; ++h, ++it) {
+                        const int b = it % kAccBufs;
+                        if (!(ok = mbar_wait(&acc_empty[b], ((it / kAccBufs) & 1) ^ 1, abort_flag))) break;
+                        tc_fence_after_sync();
+                        transform(a_addr, h == 0, 0, b);
+                        tc_commit(&acc_full[b]);
+                    }
+                    if (ok) tc_commit(&empty_bar[s]);                        // both transforms have read the stage
+                }
+            } else
             for (uint32_t t = blockIdx.x; t < num_tiles && ok; t += gridDim.x) {
                 int v = 0;
 #pragma unroll
                 for (int i = 1; i < kQuantMaxViews; ++i)
                     if (i < p.n_views && t >= p.view[i].tile_begin) v = i;
                 const bool rowwise = p.view[v].reduce_dim == 1;
-                const uint32_t idesc = idesc_k | ((rowwise ? 0u : 1u) << 15);
 #pragma unroll
                 for (int h = 0; h < KW; ++h, ++it) {                       // KW = 2: k-tile h goes through T_h into its own accumulator
                     const int s = it % kStagesQ, b = it % kAccBufs;
                     if (!(ok = mbar_wait(&acc_empty[b], ((it / kAccBufs) & 1) ^ 1, abort_flag))) break;
                     if (!(ok = mbar_wait(&full_bar[s], (it / kStagesQ) & 1, abort_flag))) break;
                     tc_fence_after_sync();
-                    const uint32_t a_addr = smem_u32(smem + s * kTileBytes);
-#pragma unroll
-                    for (int ks = 0; ks < 8; ++ks) {                       // K = 16 per MMA
-                        uint64_t adesc;
-                        if (rowwise)            // K-major: box ks/4, 32 bytes of K per step inside the 128-byte swizzle atom
-                            adesc = make_smem_desc(a_addr + (ks >> 2) * kBoxBytes + (ks & 3) * 32, 16, 1024, 2);
-                        else                    // MN-major: 16 k-rows of 128 B per step; the second 64 output rows sit one box further
-                            adesc = make_smem_desc(a_addr + ks * 2048, kBoxBytes, 1024, 2);
-                        const uint64_t bdesc = make_smem_desc(t_addr + h * kTBytes + (ks >> 2) * kBoxBytes + (ks & 3) * 32, 16, 1024, 2);
-                        tc_mma_f16(tmem_base + b * kTile, adesc, bdesc, idesc, ks != 0 ? 1u : 0u);
-                    }
+                    transform(smem_u32(smem + s * kTileBytes), rowwise, h, b);
                     tc_commit(&empty_bar[s]);
                     tc_commit(&acc_full[b]);
                 }
@@ -298,9 +332,14 @@ __device__ __forceinline__ void quantize_tc_body(const QMaps& maps, const QParam
             return (uint64_t)(pos.rt * (uint32_t)kTile + lane_row) * (uint64_t)p.view[pos.v].K + (uint64_t)(pos.kt * (uint32_t)(kTile * KW));
         };
 
+        // logical tile of this CTA's i-th accumulator: tiles are dealt out round-robin; in a DUAL launch whole units are
+        // (two consecutive logical tiles, one per view), so that both transforms of a unit read the same stage
+        auto tile_of = [&](uint32_t i) -> uint32_t {
+            return DUAL ? 2u * (blockIdx.x + (i >> 1) * gridDim.x) + (i & 1u) : blockIdx.x + i * gridDim.x;
+        };
         uint32_t it = LITE ? 0u : (uint32_t)grp;
-        uint32_t t = blockIdx.x + it * gridDim.x;
-        TilePos pos = locate_tile(p, t < num_tiles ? t : 0u);
+        uint32_t t = tile_of(it);
+        TilePos pos = DUAL ? locate_dual(p, t < num_tiles ? t : 0u) : locate_tile(p, t < num_tiles ? t : 0u);
         uint32_t rw[8];
         if (mode_draws(MODE)) view_draws32<kFold>(p.keys, p.view[pos.v].stream_tag, &p.view[pos.v].pv, first_elem(pos) + 32u * jb, rw);
         if (KW == 2) {
@@ -383,7 +422,7 @@ __device__ __forceinline__ void quantize_tc_body(const QMaps& maps, const QParam
                 if (MODE != kModeDump && live) *reinterpret_cast<uint32_t*>(scale_dst) = sb_all;
             }
         } else
-        for (; t < num_tiles; t += stride, it += (LITE ? 1 : kEpiGroups)) {
+        for (; t < num_tiles; it += (LITE ? 1 : kEpiGroups), t = DUAL ? tile_of(it) : t + stride) {
             const int b = it % kAccBufs;
             const QView& vw = p.view[pos.v];
             const uint32_t rt = pos.rt, kt = pos.kt;
@@ -399,7 +438,12 @@ __device__ __forceinline__ void quantize_tc_body(const QMaps& maps, const QParam
             const uint32_t tag_cur = vw.stream_tag;
             const PhiloxViewConsts* pv_cur = &vw.pv;
             // position of the next tile of this group (past the end: computed but not used)
-            pos = t + stride < num_tiles ? advance_tile(p, pos, t + stride) : locate_tile(p, 0u);
+            if (DUAL) {
+                const uint32_t t_next = tile_of(it + kEpiGroups);
+                pos = locate_dual(p, t_next < num_tiles ? t_next : 0u);
+            } else {
+                pos = t + stride < num_tiles ? advance_tile(p, pos, t + stride) : locate_tile(p, 0u);
+            }
             const uint64_t i_next = first_elem(pos);
             const uint32_t tag_next = p.view[pos.v].stream_tag;
             const PhiloxViewConsts* pv_next = &p.view[pos.v].pv;
@@ -470,14 +514,21 @@ __device__ __forceinline__ void quantize_tc_body(const QMaps& maps, const QParam
 template <int MODE, int KW>
 __global__ void __launch_bounds__(QCfg<false>::kThreads, 1)
 quantize_tc_kernel(const __grid_constant__ QMaps maps, const __grid_constant__ QParams p) {
-    quantize_tc_body<MODE, KW, false>(maps, p);
+    quantize_tc_body<MODE, KW, false, false>(maps, p);
+}
+
+// Both views of one tensor from one read of it (Algorithm 3 lines 3 and 5 use the same dL/dy), g <= 128.
+template <int MODE>
+__global__ void __launch_bounds__(QCfg<false>::kThreads, 1)
+quantize_tc_dual_kernel(const __grid_constant__ QMaps maps, const __grid_constant__ QParams p) {
+    quantize_tc_body<MODE, 1, false, true>(maps, p);
 }
 
 // The small-footprint build (see QCfg), g <= 128.
 template <int MODE>
 __global__ void __maxnreg__(QCfg<true>::kLaunchRegs)
 quantize_tc_lite_kernel(const __grid_constant__ QMaps maps, const __grid_constant__ QParams p) {
-    quantize_tc_body<MODE, 1, true>(maps, p);
+    quantize_tc_body<MODE, 1, true, false>(maps, p);
 }
 
 }  // namespace
@@ -518,6 +569,12 @@ cudaError_t quant_tc_init() {
         const cudaError_t e = quant_kernel_init<false>(k);
         if (e != cudaSuccess) return e;
     }
+    const void* dual[3] = {(const void*)quantize_tc_dual_kernel<kModeSR>, (const void*)quantize_tc_dual_kernel<kModeRN>,
+                           (const void*)quantize_tc_dual_kernel<kModeSR16>};
+    for (const void* k : dual) {
+        const cudaError_t e = quant_kernel_init<false>(k);
+        if (e != cudaSuccess) return e;
+    }
     const void* lite[3] = {(const void*)quantize_tc_lite_kernel<kModeSR>, (const void*)quantize_tc_lite_kernel<kModeRN>,
                            (const void*)quantize_tc_lite_kernel<kModeSR16>};
     for (const void* k : lite) {
@@ -528,8 +585,12 @@ cudaError_t quant_tc_init() {
 }
 
 // Quantise n (1..kQuantMaxViews) eligible operand views that share g, seed, rounding and scale layout in one launch.
-cudaError_t launch_quantize_tc_group(const QuantArgs* a, int n, bool dump_y, cudaStream_t stream, bool lite) {
+cudaError_t launch_quantize_tc_group(const QuantArgs* a, int n, bool dump_y, cudaStream_t stream, bool lite, bool dual) {
     if (n < 1 || n > kQuantMaxViews) return cudaErrorInvalidValue;
+    // dual: a[0] and a[1] are the row-wise and the transposed view of one tensor, whose tiles are then loaded once for both
+    if (dual && (n != 2 || lite || dump_y || a[0].g == 256 || a[0].custom_t != nullptr || a[0].x != a[1].x || a[0].rows != a[1].rows ||
+                 a[0].cols != a[1].cols || a[0].ld != a[1].ld || a[0].reduce_dim != 1 || a[1].reduce_dim != 0 || a[0].rows % kTile != 0))
+        return cudaErrorInvalidValue;
     if (lite && (dump_y || a[0].g == 256 || a[0].custom_t != nullptr)) return cudaErrorInvalidValue;   // the small build: RHT with g <= 128, quantising
     QParams p;
     QMaps maps;
@@ -568,7 +629,8 @@ cudaError_t launch_quantize_tc_group(const QuantArgs* a, int n, bool dump_y, cud
     if (e != cudaSuccess) return e;
     e = cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
     if (e != cudaSuccess) return e;
-    const unsigned grid = tiles < (uint32_t)sms ? tiles : (unsigned)sms;
+    const uint32_t units = dual ? tiles / 2 : tiles;       // loads: in a dual launch the two views' tiles pair up
+    const unsigned grid = units < (uint32_t)sms ? units : (unsigned)sms;
     for (int v = 0; v < kQuantMaxViews; ++v) {
         QView& w = p.view[v];
         w.minor_count = w.reduce_dim == 1 ? w.k_tiles : w.r_tiles;
@@ -579,7 +641,8 @@ cudaError_t launch_quantize_tc_group(const QuantArgs* a, int n, bool dump_y, cud
     }
     const bool wide = p.g == 256;
     void (*kernel)(QMaps, QParams);
-    if (lite) kernel = a[0].rounding == 0 ? quantize_tc_lite_kernel<kModeSR> : a[0].rounding == 2 ? quantize_tc_lite_kernel<kModeSR16> : quantize_tc_lite_kernel<kModeRN>;
+    if (dual) kernel = a[0].rounding == 0 ? quantize_tc_dual_kernel<kModeSR> : a[0].rounding == 2 ? quantize_tc_dual_kernel<kModeSR16> : quantize_tc_dual_kernel<kModeRN>;
+    else if (lite) kernel = a[0].rounding == 0 ? quantize_tc_lite_kernel<kModeSR> : a[0].rounding == 2 ? quantize_tc_lite_kernel<kModeSR16> : quantize_tc_lite_kernel<kModeRN>;
     else if (dump_y) kernel = wide ? quantize_tc_kernel<kModeDump, 2> : quantize_tc_kernel<kModeDump, 1>;
     else if (a[0].rounding == 0) kernel = wide ? quantize_tc_kernel<kModeSR, 2> : quantize_tc_kernel<kModeSR, 1>;
     else if (a[0].rounding == 2) kernel = wide ? quantize_tc_kernel<kModeSR16, 2> : quantize_tc_kernel<kModeSR16, 1>;
@@ -596,7 +659,7 @@ cudaError_t launch_quantize_tc_group(const QuantArgs* a, int n, bool dump_y, cud
 }
 
 cudaError_t launch_quantize_tc(const QuantArgs& a, bool dump_y, cudaStream_t stream) {
-    return launch_quantize_tc_group(&a, 1, dump_y, stream, false);
+    return launch_quantize_tc_group(&a, 1, dump_y, stream, false, false);
 }
 
 }  // namespace mx

@@ -21,7 +21,7 @@ pytestmark = pytest.mark.gpu
 
 @pytest.fixture()
 def env():
-    saved = {k: os.environ.get(k) for k in ("MXFP4_FORCE_LITE", "MXFP4_OVERLAP")}
+    saved = {k: os.environ.get(k) for k in ("MXFP4_FORCE_LITE", "MXFP4_OVERLAP", "MXFP4_DUAL_DY")}
     yield os.environ
     for k, v in saved.items():
         if v is None:
@@ -83,3 +83,33 @@ def test_overlapped_backward_gives_the_same_bits(env, mode):
             res[ov] = mx.mxfp4_linear_backward(dY, X, W, 128, 5, mx.ROUND_SR, mx.OUT_BF16)
         assert mx.mxfp4_device_status() == 0
     assert torch.equal(res["0"][0], res[mode][0]) and torch.equal(res["0"][1], res[mode][1])
+
+
+@pytest.mark.parametrize("b,m,g,rounding", [(384, 640, 128, 0), (1280, 2176, 32, 2), (256, 128, 64, 1), (2048, 4096, 128, 0)])
+def test_one_read_of_dy_gives_the_same_codes_as_two(env, b, m, g, rounding):
+    """Algorithm 3 lines 3 and 5 quantise two views of the same dL/dy; by default every 128 x 128 tile of it is loaded
+    once and transformed twice (as the K-major and as the MN-major operand).  Same codes and scales as separate passes."""
+    import torch
+    if not torch.cuda.is_available():
+        pytest.skip("no GPU")
+    from paper_2502_20586_b200 import binding as mx
+    rng = np.random.default_rng(b + m)
+    n = 264
+    dY = _dev(wl.grad_like(rng, (b, m), 1e-3, outlier_rate=1e-3))
+    X = _dev(wl.activation_like(rng, (b, n)))
+    W = _dev(wl.weight_like(rng, (m, n)))
+    env["MXFP4_FORCE_LITE"] = "0"
+    ops = {}
+    for dual in ("1", "0"):
+        env["MXFP4_DUAL_DY"] = dual
+        ws = torch.zeros(mx.mxfp4_linear_backward_workspace(b, m, n), dtype=torch.uint8, device="cuda")
+        ops[dual] = [(c.clone(), s.clone()) for c, s in mx.mxfp4_quantize_operands(dY, X, W, g, 3, rounding, workspace=ws)]
+        assert mx.mxfp4_device_status() == 0
+    for (c0, s0), (c1, s1) in zip(ops["0"], ops["1"]):
+        assert torch.equal(c0, c1) and torch.equal(s0, s1)
+    # and view by view against the stand-alone call
+    for i, (t, rd) in enumerate(((dY, 1), (W, 0), (dY, 0), (X, 0))):
+        c, s = mx.mxfp4_rht_sr_quantize(t, rd, g, 3, i + 1, rounding, mx.SF_NATIVE)
+        R, K = c.shape[0], 2 * c.shape[1]
+        valid = torch.from_numpy(hp.sf_native_offsets(R, K)).cuda()        # padding rows of the last scale tile are never written
+        assert torch.equal(c, ops["1"][i][0]) and torch.equal(s[valid], ops["1"][i][1][valid])
