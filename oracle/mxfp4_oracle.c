@@ -520,3 +520,200 @@ ORC_API int orc_num_threads(void)
     return 1;
 #endif
 }
+
+/* ========================================================================= */
+/* Extensions beyond Algorithms 1-3 (each restates a remark of the paper)     */
+/* ========================================================================= */
+
+/* ------------------------------------------------------------------------- */
+/* FP8 (E4M3) forward pass (Section 4.1, last remark; supplementary section   */
+/* "FP8 Forward Pass Results"): y = x W^T with both operands quantised to     */
+/* E4M3 under one scale per tensor, the product accumulated in high precision. */
+/* The paper names the format and the library it used, not the arithmetic;     */
+/* the reading here: scale = 448 / amax of the tensor (fp32 division; 1 for an */
+/* all-zero tensor), element = round-to-nearest-even of fp32(x * scale) onto   */
+/* the E4M3 grid, saturating at +-448, output = sum / (scale_x scale_w).       */
+/* ------------------------------------------------------------------------- */
+
+/* E4M3 ("fn": no infinities): 1 sign, 4 exponent (bias 7), 3 mantissa bits.  Exponent field 0 holds the subnormals
+ * m/8 * 2^-6; exponent field 15 with mantissa 7 is NaN, so the largest value is 1.75 * 2^8 = 448. */
+ORC_API double orc_e4m3_value(uint32_t code)
+{
+    uint32_t e = (code >> 3) & 15u, m = code & 7u;
+    double v;
+    if (e == 15u && m == 7u) return NAN;
+    if (e == 0u) v = ldexp((double)m / 8.0, -6);
+    else v = ldexp(1.0 + (double)m / 8.0, (int)e - 7);
+    return (code & 0x80u) ? -v : v;
+}
+
+/* Nearest E4M3 value of a finite v (ties to the code with even mantissa bit), saturating at +-448: found by walking
+ * the enumerated grid of the 127 non-negative finite codes 0x00..0x7E, which is increasing in the code. */
+ORC_API uint32_t orc_e4m3_round(float v)
+{
+    uint32_t sign = signbit(v) ? 0x80u : 0u;
+    double a = fabs((double)v);
+    if (!(a == a)) return 0x7Fu;
+    if (a >= 448.0) return sign | 0x7Eu;
+    uint32_t lo = 0;
+    while (lo + 1 < 0x7Fu && orc_e4m3_value(lo + 1) <= a) ++lo;       /* value(lo) <= a < value(lo + 1) */
+    double f = orc_e4m3_value(lo), c = orc_e4m3_value(lo + 1);
+    uint32_t pick;
+    if (a - f < c - a) pick = lo;
+    else if (a - f > c - a) pick = lo + 1;
+    else pick = (lo & 1u) ? lo + 1 : lo;                               /* tie: even code */
+    return sign | pick;
+}
+
+/* Scale of a bf16 tensor [R, K] (strided): 448 / amax in fp32, 1 when the tensor is all zero. */
+ORC_API float orc_fp8_tensor_scale(const uint16_t *x, int64_t R, int64_t K, int64_t stride_r, int64_t stride_k)
+{
+    float amax = 0.0f;
+    for (int64_t r = 0; r < R; ++r)
+        for (int64_t k = 0; k < K; ++k) {
+            float a = (float)fabs(bf16_to_double(x[r * stride_r + k * stride_k]));
+            if (a > amax) amax = a;
+        }
+    return amax > 0.0f ? 448.0f / amax : 1.0f;
+}
+
+/* codes[r][k] = E4M3(fp32(x[r][k] * scale)) */
+ORC_API void orc_fp8_quantize(const uint16_t *x, int64_t R, int64_t K, int64_t stride_r, int64_t stride_k, float scale,
+                              uint8_t *codes /* [R, K] */)
+{
+#pragma omp parallel for schedule(static)
+    for (int64_t r = 0; r < R; ++r)
+        for (int64_t k = 0; k < K; ++k) {
+            volatile float v = (float)bf16_to_double(x[r * stride_r + k * stride_k]) * scale;   /* one fp32 rounding */
+            codes[r * K + k] = (uint8_t)orc_e4m3_round(v);
+        }
+}
+
+/* C[i][j] = alpha sum_k value(A[i][k]) value(B[j][k]) in fp64 on the selected rows / columns (NULL = all). */
+ORC_API void orc_fp8_gemm(const uint8_t *A, const uint8_t *B, int64_t M, int64_t N, int64_t K, double alpha,
+                          const int64_t *rows, int64_t n_rows, const int64_t *cols, int64_t n_cols, double *C)
+{
+    if (!rows) n_rows = M;
+    if (!cols) n_cols = N;
+#pragma omp parallel for schedule(static)
+    for (int64_t ii = 0; ii < n_rows; ++ii) {
+        int64_t i = rows ? rows[ii] : ii;
+        for (int64_t jj = 0; jj < n_cols; ++jj) {
+            int64_t j = cols ? cols[jj] : jj;
+            double s = 0.0;
+            for (int64_t k = 0; k < K; ++k) s += orc_e4m3_value(A[i * K + k]) * orc_e4m3_value(B[j * K + k]);
+            C[ii * n_cols + jj] = alpha * s;
+        }
+    }
+}
+
+/* The forward pass y [b, m] = x [b, n] W [m, n]^T through E4M3, on the selected rows / columns of y. */
+ORC_API void orc_linear_forward_fp8(const uint16_t *x, const uint16_t *W, int64_t b, int64_t n, int64_t m,
+                                    const int64_t *rows, int64_t n_rows, const int64_t *cols, int64_t n_cols, double *y)
+{
+    float sx = orc_fp8_tensor_scale(x, b, n, n, 1), sw = orc_fp8_tensor_scale(W, m, n, n, 1);
+    uint8_t *cx = (uint8_t *)malloc((size_t)b * n), *cw = (uint8_t *)malloc((size_t)m * n);
+    orc_fp8_quantize(x, b, n, n, 1, sx, cx);
+    orc_fp8_quantize(W, m, n, n, 1, sw, cw);
+    orc_fp8_gemm(cx, cw, b, m, n, 1.0 / ((double)sx * (double)sw), rows, n_rows, cols, n_cols, y);
+    free(cx); free(cw);
+}
+
+/* ------------------------------------------------------------------------- */
+/* MXINT4 elements (Section 3, opening: "our analysis also applies to other    */
+/* low precision datatypes such as MXINT4").  The paper gives no definition;   */
+/* the reading here: an element is a 4-bit sign-magnitude integer q in          */
+/* [-7, 7], 32 elements share an E8M0 scale X, the value is q X.  The largest  */
+/* power of two among the elements is 4 = 2^2, so Algorithm 1's rule is the     */
+/* MXFP4 one, shared_exp = floor(log2 amax) - 2 (amax / X in [4, 8), values in  */
+/* (7, 8) clip under nearest rounding); Algorithm 2 pre-scales by 3/4           */
+/* (|w| < 6 <= 7) and rounds stochastically on the UNIFORM integer grid, which  */
+/* is Eq. 1-2 as printed.  The product of two such operands estimates 9/16 of   */
+/* the true product, as for MXFP4.  Code byte: bit 3 = sign, bits 0-2 = |q|.    */
+/* ------------------------------------------------------------------------- */
+
+ORC_API double orc_int4_value(uint32_t code)
+{
+    double v = (double)(code & 7u);
+    return (code & 8u) ? -v : v;
+}
+
+/* Eq. 1-2 with the dither delta = 1/2 - (r + 1/2)/256 in (-1/2, 1/2), r the 8-bit draw of the element (the draw of
+ * the MXFP4 path): ceil iff x + delta >= floor(x) + 1/2, i.e. iff 256 frac >= r + 1/2. */
+ORC_API uint32_t orc_int4_sr_round(double w, uint32_t r)
+{
+    uint32_t sign = signbit(w) ? 8u : 0u;
+    double a = fabs(w);
+    if (a >= 7.0) return sign | 7u;                       /* unreachable after the 3/4 pre-scale */
+    double fl = floor(a), delta = 0.5 - ((double)r + 0.5) / 256.0;
+    uint32_t q = (uint32_t)fl + ((a + delta >= fl + 0.5) ? 1u : 0u);
+    return sign | q;
+}
+
+/* nearest integer, ties to even, saturating at 7 (Algorithm 1 line 4 for this element format) */
+ORC_API uint32_t orc_int4_rn_round(double w)
+{
+    uint32_t sign = signbit(w) ? 8u : 0u;
+    double a = fabs(w);
+    if (a >= 7.0) return sign | 7u;
+    double fl = floor(a), fr = a - fl;
+    uint32_t q = (uint32_t)fl;
+    if (fr > 0.5 || (fr == 0.5 && (q & 1u))) ++q;
+    return sign | q;
+}
+
+/* Algorithm 2 (rounding 0) / Algorithm 1 (rounding 1) with MXINT4 elements on fp32 pre-quantisation values y [R, K];
+ * row_ids as in orc_quantize_rows.  Scale bytes follow orc_e8m0_from_amax. */
+ORC_API int orc_mxint4_quantize_rows(const float *y, int64_t R, int64_t K, int rounding, uint64_t seed, uint32_t stream_tag,
+                                     const int64_t *row_ids, uint8_t *codes, uint8_t *scales)
+{
+    if (K % 32 != 0 || (rounding != 0 && rounding != 1)) return -1;
+    const int64_t nblk = K / 32;
+#pragma omp parallel for schedule(static)
+    for (int64_t r = 0; r < R; ++r)
+        for (int64_t b = 0; b < nblk; ++b) {
+            const float *V = y + r * K + b * 32;
+            float amax = 0.0f;
+            int finite = 1;
+            for (int i = 0; i < 32; ++i) {
+                float av = fabsf(V[i]);
+                if (!(av == av) || isinf(av)) finite = 0;
+                if (av > amax) amax = av;
+            }
+            uint32_t byte = finite ? orc_e8m0_from_amax(amax) : 255u;
+            scales[r * nblk + b] = (uint8_t)byte;
+            if (byte == 255u) { memset(codes + r * K + b * 32, 0, 32); continue; }
+            int shared_exp = (int)byte - 127;
+            for (int i = 0; i < 32; ++i) {
+                int64_t elem = (row_ids ? row_ids[r] : r) * K + b * 32 + i;
+                if (rounding == 0)
+                    codes[r * K + b * 32 + i] = (uint8_t)orc_int4_sr_round(ldexp(0.75 * (double)V[i], -shared_exp),
+                                                                           orc_sr_draw(seed, stream_tag, (uint64_t)elem));
+                else
+                    codes[r * K + b * 32 + i] = (uint8_t)orc_int4_rn_round(ldexp((double)V[i], -shared_exp));
+            }
+        }
+    return 0;
+}
+
+/* C[i][j] = alpha sum_k q_A X_A q_B X_B in fp64 (the MXFP4 GEMM with integer elements) */
+ORC_API void orc_mxint4_gemm(const uint8_t *A_codes, const uint8_t *A_scales, const uint8_t *B_codes, const uint8_t *B_scales,
+                             int64_t M, int64_t N, int64_t K, double alpha,
+                             const int64_t *rows, int64_t n_rows, const int64_t *cols, int64_t n_cols, double *C)
+{
+    const int64_t nblk = K / 32;
+    if (!rows) n_rows = M;
+    if (!cols) n_cols = N;
+#pragma omp parallel for schedule(static)
+    for (int64_t ii = 0; ii < n_rows; ++ii) {
+        int64_t i = rows ? rows[ii] : ii;
+        for (int64_t jj = 0; jj < n_cols; ++jj) {
+            int64_t j = cols ? cols[jj] : jj;
+            double s = 0.0;
+            for (int64_t k = 0; k < K; ++k)
+                s += ldexp(orc_int4_value(A_codes[i * K + k]), (int)A_scales[i * nblk + k / 32] - 127) *
+                     ldexp(orc_int4_value(B_codes[j * K + k]), (int)B_scales[j * nblk + k / 32] - 127);
+            C[ii * n_cols + jj] = alpha * s;
+        }
+    }
+}

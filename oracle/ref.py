@@ -64,6 +64,28 @@ _lib.orc_linear_backward.argtypes = [_u16p, _u16p, _u16p, _i64, _i64, _i64, C.c_
 _lib.orc_linear_backward.restype = C.c_int
 _lib.orc_bias_grad.argtypes = [_u16p, _i64, _i64, _f64p]
 _lib.orc_bias_grad.restype = None
+_lib.orc_e4m3_value.argtypes = [C.c_uint32]
+_lib.orc_e4m3_value.restype = C.c_double
+_lib.orc_e4m3_round.argtypes = [C.c_float]
+_lib.orc_e4m3_round.restype = C.c_uint32
+_lib.orc_fp8_tensor_scale.argtypes = [_u16p, _i64, _i64, _i64, _i64]
+_lib.orc_fp8_tensor_scale.restype = C.c_float
+_lib.orc_fp8_quantize.argtypes = [_u16p, _i64, _i64, _i64, _i64, C.c_float, _u8p]
+_lib.orc_fp8_quantize.restype = None
+_lib.orc_fp8_gemm.argtypes = [_u8p, _u8p, _i64, _i64, _i64, C.c_double, C.c_void_p, _i64, C.c_void_p, _i64, _f64p]
+_lib.orc_fp8_gemm.restype = None
+_lib.orc_linear_forward_fp8.argtypes = [_u16p, _u16p, _i64, _i64, _i64, C.c_void_p, _i64, C.c_void_p, _i64, _f64p]
+_lib.orc_linear_forward_fp8.restype = None
+_lib.orc_int4_value.argtypes = [C.c_uint32]
+_lib.orc_int4_value.restype = C.c_double
+_lib.orc_int4_sr_round.argtypes = [C.c_double, C.c_uint32]
+_lib.orc_int4_sr_round.restype = C.c_uint32
+_lib.orc_int4_rn_round.argtypes = [C.c_double]
+_lib.orc_int4_rn_round.restype = C.c_uint32
+_lib.orc_mxint4_quantize_rows.argtypes = [_f32p, _i64, _i64, C.c_int, _u64, C.c_uint32, C.c_void_p, _u8p, _u8p]
+_lib.orc_mxint4_quantize_rows.restype = C.c_int
+_lib.orc_mxint4_gemm.argtypes = [_u8p, _u8p, _u8p, _u8p, _i64, _i64, _i64, C.c_double, C.c_void_p, _i64, C.c_void_p, _i64, _f64p]
+_lib.orc_mxint4_gemm.restype = None
 _lib.orc_num_threads.argtypes = []
 _lib.orc_num_threads.restype = C.c_int
 
@@ -243,3 +265,87 @@ def linear_backward(dY, X, W, g, rounding, seed, dx_rows=None, dx_cols=None, dw_
     if rc != 0:
         raise ValueError("bad g / shape")
     return dX, dW
+
+
+# ---------------------------------------------------------------- FP8 (E4M3) forward pass (Section 4.1 / supplementary)
+def e4m3_value(code: int) -> float:
+    return float(_lib.orc_e4m3_value(code))
+
+
+def e4m3_round(v: float) -> int:
+    return int(_lib.orc_e4m3_round(float(np.float32(v))))
+
+
+def fp8_tensor_scale(x: np.ndarray) -> float:
+    """448 / amax of a bf16 tensor (fp32), 1 for an all-zero tensor."""
+    assert x.dtype == np.uint16 and x.ndim == 2 and x.flags.c_contiguous
+    return float(_lib.orc_fp8_tensor_scale(x, x.shape[0], x.shape[1], x.shape[1], 1))
+
+
+def fp8_quantize(x: np.ndarray, scale=None):
+    """bf16 [R, K] -> (E4M3 codes [R, K], scale)."""
+    if scale is None:
+        scale = fp8_tensor_scale(x)
+    codes = np.empty(x.shape, np.uint8)
+    _lib.orc_fp8_quantize(x, x.shape[0], x.shape[1], x.shape[1], 1, scale, codes)
+    return codes, scale
+
+
+def fp8_gemm(A, B, alpha=1.0, rows=None, cols=None) -> np.ndarray:
+    M, K = A.shape
+    N, K2 = B.shape
+    assert K == K2
+    rp, nr, _r = _idx(rows)
+    cp, nc, _c = _idx(cols)
+    out = np.empty((nr if rows is not None else M, nc if cols is not None else N), np.float64)
+    _lib.orc_fp8_gemm(np.ascontiguousarray(A), np.ascontiguousarray(B), M, N, K, alpha, rp, nr, cp, nc, out)
+    return out
+
+
+def linear_forward_fp8(x, W, rows=None, cols=None) -> np.ndarray:
+    """y [b, m] = x [b, n] W [m, n]^T with E4M3 operands (one scale per tensor), fp64 accumulation."""
+    b, n = x.shape
+    m, n2 = W.shape
+    assert n == n2
+    rp, nr, _r = _idx(rows)
+    cp, nc, _c = _idx(cols)
+    out = np.empty((nr if rows is not None else b, nc if cols is not None else m), np.float64)
+    _lib.orc_linear_forward_fp8(x, W, b, n, m, rp, nr, cp, nc, out)
+    return out
+
+
+# ---------------------------------------------------------------- MXINT4 elements (Section 3, opening remark)
+def int4_value(code: int) -> float:
+    return float(_lib.orc_int4_value(code))
+
+
+def int4_sr_round(w: float, r: int) -> int:
+    return int(_lib.orc_int4_sr_round(w, r))
+
+
+def int4_rn_round(w: float) -> int:
+    return int(_lib.orc_int4_rn_round(w))
+
+
+def mxint4_quantize(y: np.ndarray, rounding: int, seed: int, stream_tag: int, row_ids=None):
+    """fp32 [R, K] -> (codes [R, K]: bit 3 sign, bits 0-2 magnitude; E8M0 scale bytes [R, K/32])."""
+    y = np.ascontiguousarray(y, np.float32)
+    R, K = y.shape
+    codes = np.empty((R, K), np.uint8)
+    scales = np.empty((R, K // 32), np.uint8)
+    rp, _n, _keep = _idx(row_ids)
+    if _lib.orc_mxint4_quantize_rows(y, R, K, rounding, seed, stream_tag, rp, codes, scales) != 0:
+        raise ValueError("K must be a multiple of 32; rounding 0 (SR) or 1 (RN)")
+    return codes, scales
+
+
+def mxint4_gemm(A_codes, A_scales, B_codes, B_scales, alpha=1.0, rows=None, cols=None) -> np.ndarray:
+    M, K = A_codes.shape
+    N, K2 = B_codes.shape
+    assert K == K2
+    rp, nr, _r = _idx(rows)
+    cp, nc, _c = _idx(cols)
+    out = np.empty((nr if rows is not None else M, nc if cols is not None else N), np.float64)
+    _lib.orc_mxint4_gemm(np.ascontiguousarray(A_codes), np.ascontiguousarray(A_scales), np.ascontiguousarray(B_codes),
+                         np.ascontiguousarray(B_scales), M, N, K, alpha, rp, nr, cp, nc, out)
+    return out
