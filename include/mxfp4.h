@@ -238,6 +238,51 @@ MXFP4_API mxfp4_status mxfp4_linear_backward_static(const void* dY, const void* 
                                                     void* dX, void* dW, int out_dtype, void* cuda_stream);
 
 /*
+ * FP8 (E4M3) forward pass (Section 4.1, closing remark, and the supplementary section "FP8 Forward Pass Results":
+ * the MXFP4 backward pass combined with an E4M3 forward pass).  y = x W^T with both operands quantised to E4M3 under
+ * one scale per tensor; the paper names the format, the arithmetic below is this library's reading of it.
+ *
+ * mxfp4_fp8_quantize: x bf16 [rows, cols] (leading dimension ld; cols and ld multiples of 8).  scale[0] receives
+ *   448 / amax(|x|) computed in fp32 (1 for an all-zero tensor), scale[1] the amax itself (it is the call's scratch
+ *   word): `scale` points to TWO floats on the device, 8-byte aligned.  codes [rows, cols] bytes receive
+ *   E4M3(fp32(x * scale[0])), round-to-nearest-even, saturating at +-448.  Two kernels, no host synchronisation.
+ * mxfp4_fp8_gemm: C [M, N] = (sum_k A[i, k] B[j, k]) / (A_scale[0] B_scale[0]); A [M, K], B [N, K] E4M3 bytes, K-major,
+ *   K % 128 == 0, N % 8 == 0; the scales are DEVICE pointers (as written by mxfp4_fp8_quantize); fp32 accumulation on the
+ *   tensor cores (tcgen05 kind::f8f6f4); C bf16 or fp32, leading dimension ldc.
+ * mxfp4_linear_forward_fp8: y [b, m] = x [b, n] W [m, n]^T through the two calls above; n % 128 == 0, m % 8 == 0;
+ *   workspace of mxfp4_linear_forward_fp8_workspace(b, n, m) bytes, 256-byte aligned (codes of both operands, scales).
+ * Errors as for the other calls (MXFP4_ERR_NULL / _SHAPE / _ALIGN / _MODE / _WORKSPACE / _CUDA).
+ */
+MXFP4_API mxfp4_status mxfp4_fp8_quantize(const void* x, int64_t rows, int64_t cols, int64_t ld, uint8_t* codes, float* scale,
+                                          void* cuda_stream);
+MXFP4_API mxfp4_status mxfp4_fp8_gemm(const uint8_t* A_codes, const float* A_scale, const uint8_t* B_codes, const float* B_scale,
+                                      int64_t M, int64_t N, int64_t K, void* C, int64_t ldc, int out_dtype, void* cuda_stream);
+MXFP4_API size_t mxfp4_linear_forward_fp8_workspace(int64_t b, int64_t n, int64_t m);
+MXFP4_API mxfp4_status mxfp4_linear_forward_fp8(const void* x, const void* W, int64_t b, int64_t n, int64_t m, void* y, int out_dtype,
+                                                void* workspace, size_t workspace_bytes, void* cuda_stream);
+
+/*
+ * MXINT4 elements (Section 3, opening: the analysis "also applies to other low precision datatypes such as MXINT4").
+ * An element is a sign-magnitude integer in [-7, 7]; 32 elements along the reduction dimension share one E8M0 scale,
+ * chosen by the rule of Algorithms 1 / 2 with emax_elem = 2 (the largest power of two among the elements is 4).
+ * MXFP4_ROUND_SR: Algorithm 2 (3/4 pre-scale, stochastic rounding on the integer grid, which is Eq. 1-2 as printed,
+ * with the 8-bit draws of the MXFP4 path); MXFP4_ROUND_RN: Algorithm 1 (nearest, ties to even, saturating at 7).
+ *
+ * mxfp4_int4_quantize: arguments as mxfp4_rht_sr_quantize (same transform, same sign vector, same draws), except:
+ *   codes [R, K] is ONE BYTE per element, the integer held as an E4M3 number (the tensor core has no 4-bit integer
+ *   type; E4M3 holds -7..7 exactly), scales always in the NATIVE layout, and y_scratch (fp32 [R, K], 16-byte
+ *   aligned, caller-owned) receives the transformed values on the way.
+ * mxfp4_int4_gemm: C [M, N] = alpha sum_k q_A X_A q_B X_B on the tensor cores (tcgen05 kind::mxf8f6f4, one scale per
+ *   32 elements); K % 128 == 0, N % 8 == 0; alpha = 16/9 undoes two 3/4 pre-scales as in Algorithm 3.
+ */
+MXFP4_API mxfp4_status mxfp4_int4_quantize(const void* x, int64_t rows, int64_t cols, int64_t ld, int reduce_dim, int g, int rounding,
+                                           uint64_t seed, uint32_t stream_tag, uint8_t* codes, uint8_t* scales, float* y_scratch,
+                                           void* cuda_stream);
+MXFP4_API mxfp4_status mxfp4_int4_gemm(const uint8_t* A_codes, const uint8_t* A_scales, const uint8_t* B_codes, const uint8_t* B_scales,
+                                       int64_t M, int64_t N, int64_t K, float alpha, void* C, int64_t ldc, int out_dtype,
+                                       void* cuda_stream);
+
+/*
  * Measurement aid, not part of the method (the paper has no counterpart): launches a kernel in which every CTA pair
  * issues `mma_per_pair` (rounded up to a multiple of 32) back-to-back 256 x 256 x 64 block-scaled FP4 tensor-core
  * instructions on operands resident in shared memory: no loads, no output.  *flop_out (HOST pointer) receives the

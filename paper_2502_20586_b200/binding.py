@@ -51,6 +51,18 @@ _lib.mxfp4_selftest_wait_expiry.argtypes = [_vp]
 _lib.mxfp4_selftest_wait_expiry.restype = _int
 _lib.mxfp4_fp4_ceiling.argtypes = [_i64, C.POINTER(C.c_int64), _vp]
 _lib.mxfp4_fp4_ceiling.restype = _int
+_lib.mxfp4_fp8_quantize.argtypes = [_vp, _i64, _i64, _i64, _vp, _vp, _vp]
+_lib.mxfp4_fp8_quantize.restype = _int
+_lib.mxfp4_fp8_gemm.argtypes = [_vp, _vp, _vp, _vp, _i64, _i64, _i64, _vp, _i64, _int, _vp]
+_lib.mxfp4_fp8_gemm.restype = _int
+_lib.mxfp4_linear_forward_fp8_workspace.argtypes = [_i64, _i64, _i64]
+_lib.mxfp4_linear_forward_fp8_workspace.restype = _sz
+_lib.mxfp4_linear_forward_fp8.argtypes = [_vp, _vp, _i64, _i64, _i64, _vp, _int, _vp, _sz, _vp]
+_lib.mxfp4_linear_forward_fp8.restype = _int
+_lib.mxfp4_int4_quantize.argtypes = [_vp, _i64, _i64, _i64, _int, _int, _int, _u64, _u32, _vp, _vp, _vp, _vp]
+_lib.mxfp4_int4_quantize.restype = _int
+_lib.mxfp4_int4_gemm.argtypes = [_vp, _vp, _vp, _vp, _i64, _i64, _i64, C.c_float, _vp, _i64, _int, _vp]
+_lib.mxfp4_int4_gemm.restype = _int
 _lib.mxfp4_scale_bytes.argtypes = [_i64, _i64, _int]
 _lib.mxfp4_scale_bytes.restype = _sz
 _lib.mxfp4_device_status.argtypes = [_vp]
@@ -62,7 +74,8 @@ EXPORTS = ["mxfp4_rht_sr_quantize", "mxfp4_rht", "mxfp4_gemm", "mxfp4_linear_bac
            "mxfp4_linear_backward", "mxfp4_linear_backward_static", "mxfp4_scale_bytes", "mxfp4_device_status", "mxfp4_status_string",
            "mxfp4_fp4_ceiling", "mxfp4_linear_backward_ex_workspace", "mxfp4_linear_backward_ex", "mxfp4_gemm_fused",
            "mxfp4_linear_backward_fused", "mxfp4_operand_layout", "mxfp4_quantize_operands", "mxfp4_transform_quantize",
-           "mxfp4_selftest_wait_expiry"]
+           "mxfp4_selftest_wait_expiry", "mxfp4_fp8_quantize", "mxfp4_fp8_gemm", "mxfp4_linear_forward_fp8_workspace",
+           "mxfp4_linear_forward_fp8", "mxfp4_int4_quantize", "mxfp4_int4_gemm"]
 
 
 class MxFp4Error(RuntimeError):
@@ -304,3 +317,67 @@ def mxfp4_fp4_ceiling(mma_per_pair: int) -> int:
 def mxfp4_device_status() -> int:
     """Synchronises the current stream and returns the status code (0 = OK, 9 = a device-side wait timed out)."""
     return int(_lib.mxfp4_device_status(_stream()))
+
+
+# ---------------------------------------------------------------- FP8 (E4M3) forward pass
+def mxfp4_fp8_quantize(x: torch.Tensor, codes=None, scale=None):
+    """x bf16 [rows, cols] -> (E4M3 codes [rows, cols] u8, scale f32[2] on the device: 448 / amax, amax)."""
+    assert x.is_cuda and x.dtype == torch.bfloat16 and x.dim() == 2 and x.stride(1) == 1
+    rows, cols = x.shape
+    if codes is None:
+        codes = torch.empty((rows, cols), dtype=torch.uint8, device=x.device)
+    if scale is None:
+        scale = torch.empty(2, dtype=torch.float32, device=x.device)
+    _check(_lib.mxfp4_fp8_quantize(_ptr(x), rows, cols, x.stride(0), _ptr(codes), _ptr(scale), _stream()))
+    return codes, scale
+
+
+def mxfp4_fp8_gemm(A_codes, A_scale, B_codes, B_scale, out_dtype: int = OUT_BF16, C_out=None):
+    """C [M, N] = A B^T / (A_scale[0] B_scale[0]) with E4M3 operands [M, K], [N, K]."""
+    M, K = A_codes.shape
+    N = B_codes.shape[0]
+    if C_out is None:
+        C_out = torch.empty((M, N), dtype=torch.float32 if out_dtype == OUT_FP32 else torch.bfloat16, device=A_codes.device)
+    _check(_lib.mxfp4_fp8_gemm(_ptr(A_codes), _ptr(A_scale), _ptr(B_codes), _ptr(B_scale), M, N, K, _ptr(C_out), C_out.stride(0),
+                               out_dtype, _stream()))
+    return C_out
+
+
+def mxfp4_linear_forward_fp8(x, W, out_dtype: int = OUT_BF16, y=None, workspace=None):
+    """y [b, m] = x [b, n] W [m, n]^T through E4M3 (one scale per tensor)."""
+    b, n = x.shape
+    m = W.shape[0]
+    for t in (x, W):
+        assert t.is_cuda and t.dtype == torch.bfloat16 and t.is_contiguous()
+    if y is None:
+        y = torch.empty((b, m), dtype=torch.float32 if out_dtype == OUT_FP32 else torch.bfloat16, device=x.device)
+    if workspace is None:
+        workspace = torch.empty(int(_lib.mxfp4_linear_forward_fp8_workspace(b, n, m)), dtype=torch.uint8, device=x.device)
+    _check(_lib.mxfp4_linear_forward_fp8(_ptr(x), _ptr(W), b, n, m, _ptr(y), out_dtype, _ptr(workspace), workspace.numel(), _stream()))
+    return y
+
+
+# ---------------------------------------------------------------- MXINT4 elements
+def mxfp4_int4_quantize(x: torch.Tensor, reduce_dim: int, g: int, seed: int, stream_tag: int = 0, rounding: int = ROUND_SR):
+    """x bf16 [rows, cols] -> (codes [R, K] u8: the integers -7..7 as E4M3 bytes, scales u8 in the native layout,
+    y fp32 [R, K]: the transformed values that were rounded)."""
+    assert x.is_cuda and x.dtype == torch.bfloat16 and x.dim() == 2 and x.stride(1) == 1
+    rows, cols = x.shape
+    R, K = (rows, cols) if reduce_dim == 1 else (cols, rows)
+    codes = torch.empty((R, K), dtype=torch.uint8, device=x.device)
+    scales = torch.zeros(mxfp4_scale_bytes(R, K, SF_NATIVE), dtype=torch.uint8, device=x.device)
+    y = torch.empty((R, K), dtype=torch.float32, device=x.device)
+    _check(_lib.mxfp4_int4_quantize(_ptr(x), rows, cols, x.stride(0), reduce_dim, g, rounding, seed, stream_tag, _ptr(codes), _ptr(scales),
+                                    _ptr(y), _stream()))
+    return codes, scales, y
+
+
+def mxfp4_int4_gemm(A_codes, A_scales, B_codes, B_scales, alpha: float = 1.0, out_dtype: int = OUT_BF16, C_out=None):
+    """C [M, N] = alpha * sum_k (q X)_A (q X)_B for MXINT4 operands [M, K], [N, K] (one byte per element)."""
+    M, K = A_codes.shape
+    N = B_codes.shape[0]
+    if C_out is None:
+        C_out = torch.empty((M, N), dtype=torch.float32 if out_dtype == OUT_FP32 else torch.bfloat16, device=A_codes.device)
+    _check(_lib.mxfp4_int4_gemm(_ptr(A_codes), _ptr(A_scales), _ptr(B_codes), _ptr(B_scales), M, N, K, alpha, _ptr(C_out), C_out.stride(0),
+                                out_dtype, _stream()))
+    return C_out

@@ -6,7 +6,7 @@ import sys
 HERE = os.path.dirname(os.path.abspath(__file__))
 CSRC = os.path.join(HERE, "csrc")
 LIB = os.path.join(HERE, "libmxfp4_b200.so")
-SOURCES = ["api.cu", "gemm.cu", "gemm_pair.cu", "gemm_fused.cu", "quantize.cu", "quantize_tc.cu", "static_workspace.cu", "fp4_ceiling.cu", "bias_grad.cu"]
+SOURCES = ["api.cu", "gemm.cu", "gemm_pair.cu", "gemm_fused.cu", "quantize.cu", "quantize_tc.cu", "static_workspace.cu", "fp4_ceiling.cu", "bias_grad.cu", "gemm_f8.cu", "variants.cu"]
 NVCC_FLAGS = ["-gencode", "arch=compute_100a,code=sm_100a", "-O3", "-lineinfo", "-std=c++17",
               "-Xcompiler", "-fPIC", "-Xcompiler", "-fvisibility=hidden", "--expt-relaxed-constexpr"]
 

@@ -65,7 +65,7 @@ mxfp4_status runtime_init() {
         if (cudaDeviceGetAttribute(&major, cudaDevAttrComputeCapabilityMajor, dev) != cudaSuccess) st = MXFP4_ERR_CUDA;
         else if (major != 10) st = MXFP4_ERR_DEVICE;
         else if (mx::gemm_init() != cudaSuccess || mx::gemm_pair_init() != cudaSuccess || mx::quant_tc_init() != cudaSuccess ||
-                 mx::gemm_fused_init() != cudaSuccess)
+                 mx::gemm_fused_init() != cudaSuccess || mx::gemm_f8_init() != cudaSuccess)
             st = MXFP4_ERR_CUDA;
         g_rt.dev_status[dev] = st;
         g_rt.dev_done[dev] = true;
@@ -159,10 +159,16 @@ mxfp4_status check_quant(const void* x, int64_t rows, int64_t cols, int64_t ld, 
     return MXFP4_OK;
 }
 
-// Tensor map over packed codes [rows, K/2] bytes: box = 128 bytes of K x box_rows rows, 128-byte swizzle.
+// Tensor map over a byte matrix [rows, row_bytes]: box = 128 bytes of a row x box_rows rows, 128-byte swizzle.
+mxfp4_status make_bytes_map(CUtensorMap* map, const uint8_t* codes, int64_t rows, int64_t row_bytes, int box_rows);
+// ... over packed E2M1 codes [rows, K/2] bytes.
 mxfp4_status make_codes_map(CUtensorMap* map, const uint8_t* codes, int64_t rows, int64_t K, int box_rows) {
-    const cuuint64_t dims[2] = {(cuuint64_t)(K / 2), (cuuint64_t)rows};
-    const cuuint64_t strides[1] = {(cuuint64_t)(K / 2)};
+    return make_bytes_map(map, codes, rows, K / 2, box_rows);
+}
+mxfp4_status make_bytes_map(CUtensorMap* map, const uint8_t* codes, int64_t rows, int64_t row_bytes, int box_rows) {
+    const int64_t K = 2 * row_bytes;
+    const cuuint64_t dims[2] = {(cuuint64_t)row_bytes, (cuuint64_t)rows};
+    const cuuint64_t strides[1] = {(cuuint64_t)row_bytes};
     const cuuint32_t box[2] = {(cuuint32_t)mx::kGemmBKBytes, (cuuint32_t)box_rows};
     const cuuint32_t elem_strides[2] = {1, 1};
     const CUresult r = g_rt.encode(map, CU_TENSOR_MAP_DATA_TYPE_UINT8, 2, const_cast<uint8_t*>(codes), dims, strides, box, elem_strides,
@@ -583,11 +589,103 @@ mxfp4_status mxfp4_quantize_operands(const void* dY, const void* X, const void* 
     return quantize_operands_impl(dY, X, W, b, m, n, g, rounding, seed, c, s, static_cast<cudaStream_t>(cuda_stream));
 }
 
+// ------------------------------------------------------------------------------------------ FP8 (E4M3) forward pass
+mxfp4_status mxfp4_fp8_quantize(const void* x, int64_t rows, int64_t cols, int64_t ld, uint8_t* codes, float* scale, void* cuda_stream) {
+    if (!x || !codes || !scale) return MXFP4_ERR_NULL;
+    if (rows <= 0 || cols <= 0 || ld < cols || cols % 8 != 0 || ld % 8 != 0) return MXFP4_ERR_SHAPE;
+    if (!aligned16(x) || !aligned16(codes) || (reinterpret_cast<uintptr_t>(scale) & 7u) != 0) return MXFP4_ERR_ALIGN;
+    const mxfp4_status st = runtime_init();
+    if (st != MXFP4_OK) return st;
+    return cuda_status(mx::launch_fp8_quantize(x, rows, cols, ld, codes, scale, static_cast<cudaStream_t>(cuda_stream)), "FP8 quantiser launch");
+}
+
+namespace {
+mxfp4_status gemm8_impl(const uint8_t* A, const uint8_t* B, const uint8_t* sfa, const uint8_t* sfb, const float* sa, const float* sb,
+                        int64_t M, int64_t N, int64_t K, float alpha, void* C, int64_t ldc, int out_dtype, cudaStream_t stream) {
+    mx::Gemm8Args a;
+    mxfp4_status st = make_bytes_map(&a.tmap_a, A, M, K, 128);
+    if (st != MXFP4_OK) return st;
+    if ((st = make_bytes_map(&a.tmap_b, B, N, K, 256)) != MXFP4_OK) return st;
+    a.block_scaled = sfa != nullptr;
+    a.sfa = sfa; a.sfb = sfb; a.scale_a = sa; a.scale_b = sb;
+    a.M = M; a.N = N; a.K = K; a.alpha = alpha; a.C = C; a.ldc = ldc; a.out_fp32 = out_dtype == MXFP4_OUT_FP32;
+    return cuda_status(mx::launch_gemm_f8(a, stream), "8-bit GEMM launch");
+}
+mxfp4_status check_gemm8(const void* A, const void* B, const void* C, int64_t M, int64_t N, int64_t K, int64_t ldc, int out_dtype) {
+    if (!A || !B || !C) return MXFP4_ERR_NULL;
+    if (M <= 0 || N <= 0 || K <= 0 || K % 128 != 0 || N % 8 != 0 || ldc < N) return MXFP4_ERR_SHAPE;
+    if (M > 0x7FFFFFFF || N > 0x7FFFFFFF || K > 0x7FFFFFFF) return MXFP4_ERR_SHAPE;
+    if (out_dtype != MXFP4_OUT_BF16 && out_dtype != MXFP4_OUT_FP32) return MXFP4_ERR_MODE;
+    if (!aligned16(A) || !aligned16(B) || !aligned16(C) || ldc % (out_dtype == MXFP4_OUT_FP32 ? 4 : 8) != 0) return MXFP4_ERR_ALIGN;
+    return MXFP4_OK;
+}
+}  // namespace
+
+mxfp4_status mxfp4_fp8_gemm(const uint8_t* A_codes, const float* A_scale, const uint8_t* B_codes, const float* B_scale, int64_t M, int64_t N,
+                            int64_t K, void* C, int64_t ldc, int out_dtype, void* cuda_stream) {
+    if (!A_scale || !B_scale) return MXFP4_ERR_NULL;
+    mxfp4_status st = check_gemm8(A_codes, B_codes, C, M, N, K, ldc, out_dtype);
+    if (st != MXFP4_OK) return st;
+    if ((st = runtime_init()) != MXFP4_OK) return st;
+    return gemm8_impl(A_codes, B_codes, nullptr, nullptr, A_scale, B_scale, M, N, K, 1.0f, C, ldc, out_dtype, static_cast<cudaStream_t>(cuda_stream));
+}
+
+size_t mxfp4_linear_forward_fp8_workspace(int64_t b, int64_t n, int64_t m) {
+    if (b <= 0 || n <= 0 || m <= 0) return 0;
+    return (size_t)(round_up(b * n, 1024) + round_up(m * n, 1024) + 1024);      // codes of x, codes of W, the two scale pairs
+}
+
+mxfp4_status mxfp4_linear_forward_fp8(const void* x, const void* W, int64_t b, int64_t n, int64_t m, void* y, int out_dtype,
+                                      void* workspace, size_t workspace_bytes, void* cuda_stream) {
+    if (!x || !W) return MXFP4_ERR_NULL;
+    mxfp4_status st = check_gemm8(x, W, y, b, m, n, m, out_dtype);                 // y [b, m] = x [b, K = n] W [m, K = n]^T
+    if (st != MXFP4_OK) return st;
+    if (workspace == nullptr || workspace_bytes < mxfp4_linear_forward_fp8_workspace(b, n, m) || (reinterpret_cast<uintptr_t>(workspace) & 255u) != 0)
+        return MXFP4_ERR_WORKSPACE;
+    if ((st = runtime_init()) != MXFP4_OK) return st;
+    cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
+    uint8_t* base = static_cast<uint8_t*>(workspace);
+    uint8_t* cx = base;
+    uint8_t* cw = cx + round_up(b * n, 1024);
+    float* sc = reinterpret_cast<float*>(cw + round_up(m * n, 1024));              // [0..1] x: scale, amax; [2..3] W
+    if ((st = cuda_status(mx::launch_fp8_quantize(x, b, n, n, cx, sc, stream), "FP8 quantiser launch (x)")) != MXFP4_OK) return st;
+    if ((st = cuda_status(mx::launch_fp8_quantize(W, m, n, n, cw, sc + 2, stream), "FP8 quantiser launch (W)")) != MXFP4_OK) return st;
+    return gemm8_impl(cx, cw, nullptr, nullptr, sc, sc + 2, b, m, n, 1.0f, y, m, out_dtype, stream);
+}
+
+// ------------------------------------------------------------------------------------------ MXINT4 elements
+mxfp4_status mxfp4_int4_quantize(const void* x, int64_t rows, int64_t cols, int64_t ld, int reduce_dim, int g, int rounding, uint64_t seed,
+                                 uint32_t stream_tag, uint8_t* codes, uint8_t* scales, float* y_scratch, void* cuda_stream) {
+    if (!codes || !scales || !y_scratch) return MXFP4_ERR_NULL;
+    mxfp4_status st = check_quant(x, rows, cols, ld, reduce_dim, g);
+    if (st != MXFP4_OK) return st;
+    if (rounding != MXFP4_ROUND_SR && rounding != MXFP4_ROUND_RN) return MXFP4_ERR_MODE;
+    if (!aligned16(codes) || !aligned16(y_scratch)) return MXFP4_ERR_ALIGN;
+    if ((st = runtime_init()) != MXFP4_OK) return st;
+    cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
+    // the transform is the MXFP4 path's own (its fp32 output, rounded once); only the element format differs
+    QuantArgs a{x, rows, cols, ld, reduce_dim, g, 0, seed, 0u, nullptr, nullptr, 0, y_scratch};
+    attach_input_map(a);
+    if ((st = cuda_status(mx::launch_rht_dump(a, stream), "transform launch")) != MXFP4_OK) return st;
+    const int64_t R = reduce_dim == 1 ? rows : cols, K = reduce_dim == 1 ? cols : rows;
+    return cuda_status(mx::launch_mxint4_quantize(y_scratch, R, K, rounding, seed, stream_tag, codes, scales, stream), "MXINT4 quantiser launch");
+}
+
+mxfp4_status mxfp4_int4_gemm(const uint8_t* A_codes, const uint8_t* A_scales, const uint8_t* B_codes, const uint8_t* B_scales, int64_t M,
+                             int64_t N, int64_t K, float alpha, void* C, int64_t ldc, int out_dtype, void* cuda_stream) {
+    if (!A_scales || !B_scales) return MXFP4_ERR_NULL;
+    mxfp4_status st = check_gemm8(A_codes, B_codes, C, M, N, K, ldc, out_dtype);
+    if (st != MXFP4_OK) return st;
+    if (!aligned16(A_scales) || !aligned16(B_scales)) return MXFP4_ERR_ALIGN;
+    if ((st = runtime_init()) != MXFP4_OK) return st;
+    return gemm8_impl(A_codes, B_codes, A_scales, B_scales, nullptr, nullptr, M, N, K, alpha, C, ldc, out_dtype, static_cast<cudaStream_t>(cuda_stream));
+}
+
 mxfp4_status mxfp4_device_status(void* cuda_stream) {
     if (cudaStreamSynchronize(static_cast<cudaStream_t>(cuda_stream)) != cudaSuccess) return MXFP4_ERR_CUDA;
     unsigned int word = 0;
     cudaError_t (*const fetch[])(unsigned int*) = {mx::fetch_gemm_status, mx::fetch_gemm_pair_status, mx::fetch_quant_tc_status,
-                                                   mx::fetch_fp4_ceiling_status, mx::fetch_gemm_fused_status};
+                                                   mx::fetch_fp4_ceiling_status, mx::fetch_gemm_fused_status, mx::fetch_gemm_f8_status};
     for (auto f : fetch) {
         unsigned int w = 0;
         if (f(&w) != cudaSuccess) return MXFP4_ERR_CUDA;

@@ -91,6 +91,36 @@ cudaError_t launch_gemm_fused(const FusedGemmArgs& a, cudaStream_t stream);
 cudaError_t gemm_fused_init();
 cudaError_t fetch_gemm_fused_status(unsigned int* word);
 
+// GEMM on 8-bit element containers (gemm_f8.cu): E4M3 operands with per-tensor scales (FP8 forward pass), or E4M3
+// containers of MXINT4 integers with one UE8M0 scale per 32 elements (native scale layout, K % 128 == 0).
+struct Gemm8Args {
+    CUtensorMap tmap_a;   // bytes [M, K], box 128 B x 128 rows, 128-byte swizzle
+    CUtensorMap tmap_b;   // bytes [N, K], box 128 B x 256 rows
+    bool block_scaled;
+    const uint8_t* sfa;   // block_scaled: native scale layout
+    const uint8_t* sfb;
+    const float* scale_a; // plain: device pointers to the per-tensor scales; C = A B^T / (scale_a scale_b)
+    const float* scale_b;
+    int64_t M, N, K;
+    float alpha;          // block_scaled only
+    void* C;
+    int64_t ldc;
+    int out_fp32;
+};
+cudaError_t launch_gemm_f8(const Gemm8Args& a, cudaStream_t stream);
+cudaError_t gemm_f8_init();
+cudaError_t fetch_gemm_f8_status(unsigned int* word);
+
+// Element-wise kernels of the extensions (variants.cu).
+// Per-tensor E4M3 quantisation: *scale = 448 / amax(x) (1 for an all-zero tensor), codes = E4M3(x * scale).
+// `scale` doubles as the amax scratch word while the call runs.
+cudaError_t launch_fp8_quantize(const void* x, int64_t rows, int64_t cols, int64_t ld, uint8_t* codes, float* scale, cudaStream_t stream);
+// MXINT4 from fp32 pre-quantisation values y [R, K]: per 32-block E8M0 scale (Algorithm 1 / 2 rule), elements rounded
+// to integers in [-7, 7] (rounding 0: 3/4 pre-scale + stochastic rounding with the path's Philox draws; 1: nearest),
+// stored as E4M3 bytes; scales in the native layout.
+cudaError_t launch_mxint4_quantize(const float* y, int64_t R, int64_t K, int rounding, uint64_t seed, uint32_t stream_tag,
+                                   uint8_t* codes, uint8_t* scales, cudaStream_t stream);
+
 cudaError_t launch_gemm(const GemmArgs& a, cudaStream_t stream);
 cudaError_t gemm_init();            // one-time: opt in to large dynamic shared memory
 cudaError_t launch_gemm_pair(const GemmArgs& a, cudaStream_t stream);

@@ -158,3 +158,26 @@ def test_header_is_plain_c(tmp_path):
     src.write_text('#include "include/mxfp4.h"\nint main(void) { return (int)MXFP4_ROUND_SR16 + (int)MXFP4_ERR_TIMEOUT; }\n')
     for cmd in (["gcc", "-std=c99", "-Wall", "-Wextra", "-pedantic", "-Werror"], ["g++", "-std=c++11", "-Wall", "-Wextra", "-Werror", "-x", "c++"]):
         subprocess.run(cmd + ["-I", ROOT, "-fsyntax-only", str(src)], check=True)
+
+
+def test_extension_calls_reject_bad_arguments_before_touching_the_device():
+    """FP8 forward and MXINT4 entry points: the same error discipline as the main calls (no GPU needed)."""
+    from paper_2502_20586_b200 import binding as mx
+    raw = mx.lib()
+    P = 4096                                                        # any 16-byte aligned non-null address: never dereferenced
+    assert raw.mxfp4_fp8_quantize(None, 8, 64, 64, P, P, 0) == 1
+    assert raw.mxfp4_fp8_quantize(P, 8, 60, 64, P, P, 0) == 2       # cols % 8
+    assert raw.mxfp4_fp8_quantize(P, 8, 64, 64, P, P + 4, 0) == 3   # the scale pair must be 8-byte aligned
+    assert raw.mxfp4_fp8_gemm(P, None, P, P, 128, 8, 128, P, 8, 0, 0) == 1
+    assert raw.mxfp4_fp8_gemm(P, P, P, P, 128, 8, 96, P, 8, 0, 0) == 2      # K % 128
+    assert raw.mxfp4_fp8_gemm(P, P, P, P, 128, 8, 128, P, 8, 7, 0) == 5
+    assert raw.mxfp4_linear_forward_fp8_workspace(0, 1, 1) == 0
+    need = raw.mxfp4_linear_forward_fp8_workspace(256, 512, 384)
+    assert need >= 256 * 512 + 384 * 512 + 16
+    assert raw.mxfp4_linear_forward_fp8(P, P, 256, 512, 384, P, 0, P, need - 1, 0) == 6
+    assert raw.mxfp4_linear_forward_fp8(P, P, 256, 500, 384, P, 0, P, need, 0) == 2
+    assert raw.mxfp4_int4_quantize(P, 128, 256, 256, 1, 64, 2, 0, 0, P, P, P, 0) == 5      # the 16-bit dither is an MXFP4 mode
+    assert raw.mxfp4_int4_quantize(P, 128, 256, 256, 1, 48, 0, 0, 0, P, P, P, 0) == 4
+    assert raw.mxfp4_int4_quantize(P, 128, 256, 256, 1, 64, 0, 0, 0, P, P, None, 0) == 1
+    assert raw.mxfp4_int4_gemm(P, None, P, P, 128, 8, 128, 1.0, P, 8, 0, 0) == 1
+    assert raw.mxfp4_int4_gemm(P, P, P, P, 128, 12, 128, 1.0, P, 12, 0, 0) == 2
