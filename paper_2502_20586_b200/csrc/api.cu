@@ -392,7 +392,8 @@ struct Overlap {
     bool forked = false;  // the side stream holds work that the caller's stream has to wait for
 };
 mxfp4_status quantize_operands_impl(const void* dY, const void* X, const void* W, int64_t b, int64_t m, int64_t n, int g, int rounding,
-                                    uint64_t seed, uint8_t* const c[4], uint8_t* const s[4], cudaStream_t stream, Overlap* ov = nullptr) {
+                                    uint64_t seed, uint8_t* const c[4], uint8_t* const s[4], cudaStream_t stream, Overlap* ov = nullptr,
+                                    float* col_sums = nullptr, bool* col_sums_done = nullptr) {
     QuantArgs q[4] = {
         {dY, b, m, m, 1, g, rounding, seed, 1u, c[0], s[0], 1, nullptr},   // dY   [b, K = m]
         {W, m, n, n, 0, g, rounding, seed, 2u, c[1], s[1], 1, nullptr},    // W^T  [n, K = m]
@@ -422,7 +423,8 @@ mxfp4_status quantize_operands_impl(const void* dY, const void* X, const void* W
     if (all_tc && g != 256 && !force_lite() && dual_setting()) {
         // dL/dy feeds lines 3 and 5: its two views come from ONE read of it; W^T and X^T in a second launch
         const QuantArgs dy[2] = {q[0], q[2]}, wx[2] = {q[1], q[3]};
-        if (cuda_status(mx::launch_quantize_tc_group(dy, 2, false, stream, false, true), "quantiser launch (both views of dY)") != MXFP4_OK) return MXFP4_ERR_CUDA;
+        if (cuda_status(mx::launch_quantize_tc_group(dy, 2, false, stream, false, true, col_sums), "quantiser launch (both views of dY)") != MXFP4_OK) return MXFP4_ERR_CUDA;
+        if (col_sums != nullptr && col_sums_done != nullptr) *col_sums_done = true;     // the bias gradient's first pass rode along
         return cuda_status(mx::launch_quantize_tc_group(wx, 2, false, stream), "quantiser launch (W, X)");
     }
     if (all_tc)                                     // the four views of the call in one launch
@@ -487,7 +489,9 @@ mxfp4_status linear_backward_impl(const void* dY, const void* X, const void* W, 
         const int64_t head_dx = b * m + n * m, head_dw = m * b + n * b;       // elements quantised before the first GEMM can start
         ov.first = overlap_mode == 2 ? 0 : overlap_mode == 3 ? 1 : (head_dx <= head_dw ? 0 : 1);
     }
-    if ((st = quantize_operands_impl(dY, X, W, b, m, n, g, rounding, seed, c, s, stream, &ov)) != MXFP4_OK) {
+    float* bias_partial = db != nullptr ? reinterpret_cast<float*>(base + bias_off) : nullptr;
+    bool bias_fused = false;
+    if ((st = quantize_operands_impl(dY, X, W, b, m, n, g, rounding, seed, c, s, stream, &ov, bias_partial, &bias_fused)) != MXFP4_OK) {
         if (ov.forked && (cudaEventRecord(fj->join, fj->side) != cudaSuccess || cudaStreamWaitEvent(stream, fj->join, 0) != cudaSuccess)) return MXFP4_ERR_CUDA;
         return st;
     }
@@ -507,8 +511,10 @@ mxfp4_status linear_backward_impl(const void* dY, const void* X, const void* W, 
         if (st == MXFP4_OK) st = gemm_launch(gw, fj != nullptr ? fj->side : stream);
     }
     // dL/db = 1 dL/dy (problem statement): column sums of dY, after the GEMMs on the caller's stream
+    // (when the dual-view quantiser launch has already summed every 128-row band of dY, only the bands remain to be added)
     if (st == MXFP4_OK && db != nullptr)
-        st = cuda_status(mx::launch_bias_grad(dY, b, m, m, accumulate, db, reinterpret_cast<float*>(base + bias_off), stream), "bias gradient launch");
+        st = bias_fused ? cuda_status(mx::launch_bias_finish(bias_partial, m, (int)(b / 128), accumulate, db, stream), "bias gradient launch")
+                        : cuda_status(mx::launch_bias_grad(dY, b, m, m, accumulate, db, bias_partial, stream), "bias gradient launch");
     // The join is made whatever happened after the fork, so that the side stream never runs unordered with the caller's.
     if (fj != nullptr && (cudaEventRecord(fj->join, fj->side) != cudaSuccess || cudaStreamWaitEvent(stream, fj->join, 0) != cudaSuccess))
         return MXFP4_ERR_CUDA;

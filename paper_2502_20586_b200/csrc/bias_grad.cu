@@ -66,7 +66,17 @@ int bias_grad_splits(int64_t b, int64_t m) {
     return (int)splits;
 }
 
-size_t bias_grad_workspace(int64_t b, int64_t m) { return (size_t)bias_grad_splits(b, m) * (size_t)m * sizeof(float); }
+// Room for either form of the first pass: the stand-alone kernel's splits, or one partial row per 128-row band of dY
+// when the quantiser launch computes the sums on its way.
+size_t bias_grad_workspace(int64_t b, int64_t m) {
+    const int64_t bands = (b + 127) / 128, splits = bias_grad_splits(b, m);
+    return (size_t)(bands > splits ? bands : splits) * (size_t)m * sizeof(float);
+}
+
+cudaError_t launch_bias_finish(const float* partial, int64_t m, int bands, int accumulate, float* db, cudaStream_t stream) {
+    colsum_finish<<<(unsigned)((m + 255) / 256), 256, 0, stream>>>(partial, m, bands, accumulate, db);
+    return cudaGetLastError();
+}
 
 cudaError_t launch_bias_grad(const void* dY, int64_t b, int64_t m, int64_t ld, int accumulate, float* db, float* partial, cudaStream_t stream) {
     const int splits = bias_grad_splits(b, m);

@@ -31,7 +31,9 @@ cudaError_t launch_quantize_tc(const QuantArgs& a, bool dump_y, cudaStream_t str
 constexpr int kQuantMaxViews = 4;
 // lite: the small-footprint build (g <= 128) that can share an SM with the small build of the pair GEMM.
 // dual: n = 2, a[0] / a[1] = the row-wise and the transposed view of ONE tensor (both extents multiples of 128): every tile of it is read once.
-cudaError_t launch_quantize_tc_group(const QuantArgs* a, int n, bool dump_y, cudaStream_t stream, bool lite = false, bool dual = false);
+// col_sums (dual only, may be null): fp32 [rows / 128, cols] receives the column sums of every 128-row band of that tensor.
+cudaError_t launch_quantize_tc_group(const QuantArgs* a, int n, bool dump_y, cudaStream_t stream, bool lite = false, bool dual = false,
+                                     float* col_sums = nullptr);
 
 cudaError_t launch_quantize(const QuantArgs& a, cudaStream_t stream);
 cudaError_t launch_rht_dump(const QuantArgs& a, cudaStream_t stream);
@@ -62,6 +64,9 @@ constexpr int kGemmBKBytes = 128;   // 256 E2M1 elements per pipeline stage
 // bias_grad_workspace(b, m) bytes.
 size_t bias_grad_workspace(int64_t b, int64_t m);
 cudaError_t launch_bias_grad(const void* dY, int64_t b, int64_t m, int64_t ld, int accumulate, float* db, float* partial, cudaStream_t stream);
+// Second pass alone: db [m] = (accumulate ? db : 0) + the `bands` rows of partial [bands, m] added in order (the first pass
+// was done by the dual-view quantiser launch, which holds every tile of dY in shared memory anyway).
+cudaError_t launch_bias_finish(const float* partial, int64_t m, int bands, int accumulate, float* db, cudaStream_t stream);
 
 // Each kernel file keeps its own device status word (set when a bounded wait expires); these read and clear them.
 cudaError_t fetch_gemm_status(unsigned int* word);

@@ -83,6 +83,7 @@ struct QParams {
     int g, sf_native;
     const uint16_t* custom_t;  // bf16 [g, g] row-major transform matrix given by the caller, or null (then diag(S) H_g / sqrt(g))
     uint64_t seed;
+    float* col_sums;           // DUAL launches: partial column sums [x rows / 128][x cols] of x in fp32 (bias gradient), or null
     PipeConsts pipe;           // see quant_math.cuh: constants kept opaque to the compiler
     PhiloxKeys keys;           // the ten Philox round keys of `seed` (key schedule only; the rounds run on the device)
 };
@@ -174,7 +175,9 @@ __device__ __forceinline__ void quantize_tc_body(const QMaps& maps, const QParam
     constexpr bool kFold = MODE == kModeSR16 && KW == 1;
 
     if (threadIdx.x == 0) {
-        for (int s = 0; s < kStagesQ; ++s) { mbar_init(&full_bar[s], 1); mbar_init(&empty_bar[s], 1); }
+        // a stage is free when its transforms have read it (one commit) and, with column sums on, the two summing warps too
+        const uint32_t n_readers = (DUAL && p.col_sums != nullptr) ? 3u : 1u;
+        for (int s = 0; s < kStagesQ; ++s) { mbar_init(&full_bar[s], 1); mbar_init(&empty_bar[s], n_readers); }
         for (int b = 0; b < kAccBufs; ++b) { mbar_init(&acc_full[b], 1); mbar_init(&acc_empty[b], (KW == 2 || LITE) ? 8 : 4); }
         *abort_flag = 0;
         mbar_fence_init();
@@ -308,6 +311,35 @@ __device__ __forceinline__ void quantize_tc_body(const QMaps& maps, const QParam
             }
             if (!ok) *abort_flag = 1;
         }
+    } else if (DUAL && p.col_sums != nullptr) {
+        // ------------------------------------------------------------------ warps 2, 3: column sums of the x tile (dL/db = 1 dL/dy)
+        // The tile is in shared memory anyway: warp w sums columns 64 w .. 64 w + 63 (one TMA box), a lane two adjacent
+        // columns (one 32-bit word per row; the 128-byte swizzle permutes 16-byte chunks inside a row, so a warp's 32
+        // words of a row still fall into 32 different banks), rows in order: a fixed summation order.  One partial sum
+        // per (128-row band of x, column); a second kernel adds the bands in order.
+        const int w = warp - 2;
+        uint32_t is = 0;
+        bool ok = true;
+        for (uint32_t u = blockIdx.x; 2u * u < num_tiles; u += gridDim.x, ++is) {
+            const int s = is % kStagesQ;
+            ok = mbar_wait(&full_bar[s], (is / kStagesQ) & 1, abort_flag);
+            ok = __all_sync(0xffffffffu, ok);
+            if (!ok) break;
+            const uint8_t* box = smem + s * kTileBytes + w * kBoxBytes;
+            float s0 = 0.f, s1 = 0.f;
+#pragma unroll 8
+            for (int r = 0; r < kTile; ++r) {
+                const uint32_t v = *reinterpret_cast<const uint32_t*>(box + r * 128 + ((((lane >> 2) ^ (r & 7)) << 4) | ((lane & 3) << 2)));
+                s0 += __uint_as_float(v << 16);
+                s1 += __uint_as_float(v & 0xFFFF0000u);
+            }
+            __syncwarp();
+            if (lane == 0) mbar_arrive(&empty_bar[s]);                   // this warp is done with the stage
+            const uint32_t xc_tiles = p.view[0].k_tiles, xr = u / xc_tiles, xc = u - xr * xc_tiles;
+            float* dst = p.col_sums + (int64_t)xr * p.view[0].K + (int64_t)xc * kTile + w * 64 + 2 * lane;
+            *reinterpret_cast<float2*>(dst) = make_float2(s0, s1);
+        }
+        if (!ok && lane == 0) *abort_flag = 1;
     }
     } else {
         // ------------------------------------------------------------------ epilogue (warp groups 1..4)
@@ -585,7 +617,7 @@ cudaError_t quant_tc_init() {
 }
 
 // Quantise n (1..kQuantMaxViews) eligible operand views that share g, seed, rounding and scale layout in one launch.
-cudaError_t launch_quantize_tc_group(const QuantArgs* a, int n, bool dump_y, cudaStream_t stream, bool lite, bool dual) {
+cudaError_t launch_quantize_tc_group(const QuantArgs* a, int n, bool dump_y, cudaStream_t stream, bool lite, bool dual, float* col_sums) {
     if (n < 1 || n > kQuantMaxViews) return cudaErrorInvalidValue;
     // dual: a[0] and a[1] are the row-wise and the transposed view of one tensor, whose tiles are then loaded once for both
     if (dual && (n != 2 || lite || dump_y || a[0].g == 256 || a[0].custom_t != nullptr || a[0].x != a[1].x || a[0].rows != a[1].rows ||
@@ -615,6 +647,8 @@ cudaError_t launch_quantize_tc_group(const QuantArgs* a, int n, bool dump_y, cud
     p.g = a[0].g; p.sf_native = a[0].sf_native; p.seed = a[0].seed;
     p.custom_t = static_cast<const uint16_t*>(a[0].custom_t);
     if (p.custom_t != nullptr && p.g == 256) return cudaErrorInvalidValue;
+    if (col_sums != nullptr && !dual) return cudaErrorInvalidValue;
+    p.col_sums = col_sums;
     p.pipe = make_pipe_consts();
     {   // Philox key schedule: key_i = key_0 + i * (0x9E3779B9, 0xBB67AE85)
         uint32_t k0 = (uint32_t)p.seed, k1 = (uint32_t)(p.seed >> 32);
@@ -659,7 +693,7 @@ cudaError_t launch_quantize_tc_group(const QuantArgs* a, int n, bool dump_y, cud
 }
 
 cudaError_t launch_quantize_tc(const QuantArgs& a, bool dump_y, cudaStream_t stream) {
-    return launch_quantize_tc_group(&a, 1, dump_y, stream, false, false);
+    return launch_quantize_tc_group(&a, 1, dump_y, stream, false, false, nullptr);
 }
 
 }  // namespace mx

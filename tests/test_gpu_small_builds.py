@@ -113,3 +113,27 @@ def test_one_read_of_dy_gives_the_same_codes_as_two(env, b, m, g, rounding):
         R, K = c.shape[0], 2 * c.shape[1]
         valid = torch.from_numpy(hp.sf_native_offsets(R, K)).cuda()        # padding rows of the last scale tile are never written
         assert torch.equal(c, ops["1"][i][0]) and torch.equal(s[valid], ops["1"][i][1][valid])
+
+
+def test_bias_sums_from_the_quantiser_launch_agree_with_the_separate_pass(env, ref):
+    """The bias gradient's first pass (column sums of every 128-row band of dL/dy) rides along in the dual-view quantiser
+    launch, which has every tile in shared memory anyway; with MXFP4_DUAL_DY=0 a stand-alone kernel reads dL/dy again.
+    Both against the fp64 oracle within the fp32 summation bound; dX and dW are the same bits either way."""
+    import torch
+    if not torch.cuda.is_available():
+        pytest.skip("no GPU")
+    from paper_2502_20586_b200 import binding as mx
+    rng = np.random.default_rng(77)
+    b, m, n = 2048, 1152, 264
+    dYb = wl.grad_like(rng, (b, m), 1e-3, outlier_rate=1e-3)
+    dY, X, W = _dev(dYb), _dev(wl.activation_like(rng, (b, n))), _dev(wl.weight_like(rng, (m, n)))
+    want = ref.bias_grad(dYb)
+    bound = 64 * np.sqrt(b) * 2.0 ** -24 * np.abs(wl.bf16_bits_to_f64(dYb)).sum(axis=0)
+    env["MXFP4_FORCE_LITE"] = "0"
+    res = {}
+    for dual in ("1", "0"):
+        env["MXFP4_DUAL_DY"] = dual
+        res[dual] = mx.mxfp4_linear_backward_ex(dY, X, W, 128, 5, mx.ROUND_SR, mx.OUT_FP32, with_bias=True)
+        assert mx.mxfp4_device_status() == 0
+        assert np.all(np.abs(res[dual][2].cpu().numpy().astype(np.float64) - want) <= bound)
+    assert torch.equal(res["0"][0], res["1"][0]) and torch.equal(res["0"][1], res["1"][1])
