@@ -276,7 +276,9 @@ def run_gpu(args):
             for (layer, dY, X, W, dX, dW), (wsl, ops) in zip(data, bufs):
                 fn = lambda dY=dY, X=X, W=W, wsl=wsl: mx.mxfp4_quantize_operands(dY, X, W, g, seed, rnd, workspace=wsl)
                 if record:
-                    timed("quant", layer.name, (2 * dY.numel() + X.numel() + W.numel()) * QUANT_BYTES_PER_ELEM, fn)
+                    # work = (algorithmic bytes with dL/dy read once for its two views, bytes if every view were a pass of its own)
+                    views = 2 * dY.numel() + X.numel() + W.numel()
+                    timed("quant", layer.name, ((dY.numel() + X.numel() + W.numel()) * 2.0 + views * (0.5 + 1.0 / 32.0), views * QUANT_BYTES_PER_ELEM), fn)
                 else:
                     fn()
                 for (a, bb, out, fl) in ((0, 1, dX, 2 * layer.b * layer.n * layer.m), (2, 3, dW, 2 * layer.m * layer.n * layer.b)):
@@ -301,22 +303,28 @@ def run_gpu(args):
         roof_burst = roof_leg_s < 1.0
         fp4_peak = BF16_TO_FP4 * (peaks["bf16_burst"] if roof_burst else peaks["bf16_sustained"])
         agg = {}
+        quant_per_view_bytes = 0.0
         for kind, name, a, b, work in records:
             d = agg.setdefault(kind, [0.0, 0.0, 0])
+            if kind == "quant":
+                quant_per_view_bytes += work[1]
+                work = work[0]
             d[0] += a.elapsed_time(b) * 1e-3; d[1] += work; d[2] += 1
         # the three lines per layer: quantiser alone (GB/s, of HBM peak), GEMMs alone on the quantised operands
         # (TFLOP/s, of the FP4 peaks), and the layer end to end = 4bmn / (its three launches)
         per_layer = {}
         for kind, name, a, b, work in records:
-            d = per_layer.setdefault(name, {"quant_s": 0.0, "quant_bytes": 0.0, "gemm_s": 0.0, "flops": 0.0})
+            d = per_layer.setdefault(name, {"quant_s": 0.0, "quant_bytes": 0.0, "quant_view_bytes": 0.0, "gemm_s": 0.0, "flops": 0.0})
             t = a.elapsed_time(b) * 1e-3
             if kind == "quant":
-                d["quant_s"] += t; d["quant_bytes"] += work
+                d["quant_s"] += t; d["quant_bytes"] += work[0]; d["quant_view_bytes"] += work[1]
             else:
                 d["gemm_s"] += t; d["flops"] += work
         for name, d in per_layer.items():
             q_gbs, g_tf = d["quant_bytes"] / d["quant_s"] / 1e9, d["flops"] / d["gemm_s"] / 1e12
             per_layer[name] = {"quant_GB/s": q_gbs, "quant_frac_of_hbm_peak": q_gbs / peaks["hbm_gbs"],
+                               "quant_per_view_GB/s": d["quant_view_bytes"] / d["quant_s"] / 1e9,
+                               "quant_per_view_frac_of_hbm_peak": d["quant_view_bytes"] / d["quant_s"] / 1e9 / peaks["hbm_gbs"],
                                "gemm_TFLOP/s": g_tf, "gemm_frac_of_4x_bf16_burst": g_tf / (BF16_TO_FP4 * peaks["bf16_burst"]),
                                "gemm_frac_of_nominal_9pf": g_tf / NOMINAL_FP4_TFLOPS,
                                "layer_TFLOP/s": d["flops"] / (d["quant_s"] + d["gemm_s"]) / 1e12,
@@ -329,7 +337,10 @@ def run_gpu(args):
         t_, by, n_ = agg["quant"]
         kernels["quant"] = {"launches": n_, "avg_ms": t_ / n_ * 1e3, "GB/s": by / t_ / 1e9,
                             "frac_of_hbm_peak": by / t_ / 1e9 / peaks["hbm_gbs"],
-                            "what": "the four operand views of a layer in one launch (dY row-wise and transposed, W and X transposed)"}
+                            "per_view_GB/s": quant_per_view_bytes / t_ / 1e9, "per_view_frac_of_hbm_peak": quant_per_view_bytes / t_ / 1e9 / peaks["hbm_gbs"],
+                            "what": ("the four operand views of a layer (dY row-wise and transposed, W and X transposed), one or two launches; GB/s = algorithmic "
+                                     "bytes with dL/dy read ONCE for its two views (2 B per input element + 0.53125 B per output element) / time; per_view = the bytes "
+                                     "of four separate passes (2.53125 B per view element) / time, the figure comparable with a single-view launch")}
         kernels["gemm"] = {"launches": gemm_n, "avg_ms": gemm_t / gemm_n * 1e3, "TFLOP/s": gemm_tflops,
                            "frac_of_4x_bf16_burst": gemm_tflops / (BF16_TO_FP4 * peaks["bf16_burst"]),
                            "frac_of_4x_bf16_sustained": gemm_tflops / (BF16_TO_FP4 * peaks["bf16_sustained"]),
@@ -539,7 +550,7 @@ def run_gpu(args):
                        "frac_of_nominal_9pf": value / world / NOMINAL_FP4_TFLOPS, "timed_region_s": ms * args.steps * 1e-3,
                        "step_as_separate_calls_ms": calls_ms},
             "e2e": {"value": e2e_value, "unit": UNIT, "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h, "ms_per_step": ms_e2e},
-            "gpu_launches": args.steps * len(layers) * 3,     # per layer: one grouped quantiser launch + two GEMMs
+            "gpu_launches": args.steps * sum(4 if l.b * l.m >= (1 << 25) else 3 for l in layers),   # per layer: one or two quantiser launches + two GEMMs
             "clocks": clocks,
             "roofline": None if gemm_tflops is None else {
                          "kernel": "gemm_mxf4_pair_kernel", "bound": "tensor", "achieved": gemm_tflops, "peak": fp4_peak, "unit": "TFLOP/s",

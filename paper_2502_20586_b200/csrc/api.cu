@@ -124,10 +124,12 @@ bool force_lite() {
     return e != nullptr && e[0] == '1';
 }
 
-// MXFP4_DUAL_DY=0: quantise the two views of dY as separate tile lists (two reads of dY) instead of one read for both.
-bool dual_setting() {
+// MXFP4_DUAL_DY: 1 (default) = one read of dL/dy for its two views where that pays (large layers, or a bias gradient
+// wanted); 0 = always separate tile lists (two reads); 2 = always one read.
+int dual_setting() {
     const char* e = getenv("MXFP4_DUAL_DY");
-    return !(e != nullptr && e[0] == '0');
+    if (e == nullptr || e[0] == '\0') return 1;
+    return e[0] >= '0' && e[0] <= '2' ? e[0] - '0' : 1;
 }
 
 int overlap_setting() {
@@ -420,7 +422,10 @@ mxfp4_status quantize_operands_impl(const void* dY, const void* X, const void* W
         return cuda_status(mx::launch_quantize_tc_group(tail, 2, false, ov->fj->side, true), "small quantiser launch (second product)");
     }
     if (ov != nullptr) ov->first = -1;
-    if (all_tc && g != 256 && !force_lite() && dual_setting()) {
+    // (worth a second launch only when dL/dy is large: below 2^25 elements, or when the column sums are not wanted from
+    // it either, the four views go as one tile list in one launch, which is what the small layers' short kernels prefer)
+    const int dual_mode = dual_setting();
+    if (all_tc && g != 256 && !force_lite() && (dual_mode == 2 || (dual_mode == 1 && (b * m >= (int64_t(1) << 25) || col_sums != nullptr)))) {
         // dL/dy feeds lines 3 and 5: its two views come from ONE read of it; W^T and X^T in a second launch
         const QuantArgs dy[2] = {q[0], q[2]}, wx[2] = {q[1], q[3]};
         if (cuda_status(mx::launch_quantize_tc_group(dy, 2, false, stream, false, true, col_sums), "quantiser launch (both views of dY)") != MXFP4_OK) return MXFP4_ERR_CUDA;
