@@ -386,6 +386,28 @@ def run_gpu(args):
             ms_ser, ms_ovl = sorted(ab["0"])[1], sorted(ab["1"])[1]
             variants["overlapped"] = {"ms_per_step": ms_ovl, "value": flops_step / (ms_ovl * 1e-3) / 1e12, "serial_ms_per_step_same_leg": ms_ser,
                                       "steps": k_var, "note": "median of three alternating runs of the overlapped and the serial form; the default is the serial form"}
+        # the E4M3 forward pass the MXFP4 backward is compatible with (Section 4.1): y = x W^T of the same four layers
+        if all(l.n % 128 == 0 and l.m % 8 == 0 for l in layers):
+            fwd = [(X, W, torch.empty((l.b, l.m), dtype=torch.bfloat16, device=dev),
+                    torch.empty(int(mx.lib().mxfp4_linear_forward_fp8_workspace(l.b, l.n, l.m)), dtype=torch.uint8, device=dev))
+                   for (l, dY, X, W, dX, dW) in data]
+
+            def step_fwd():
+                for (X, W, y, wsf) in fwd:
+                    mx.mxfp4_linear_forward_fp8(X, W, out_dtype, y=y, workspace=wsf)
+            step_fwd()
+            a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            k_var = max(1, min(args.steps, 10))
+            barrier()
+            a.record(stream)
+            for _ in range(k_var):
+                step_fwd()
+            b.record(stream)
+            barrier()
+            ms_var = a.elapsed_time(b) / k_var
+            variants["fp8_forward"] = {"ms_per_step": ms_var, "value": 0.5 * flops_step / (ms_var * 1e-3) / 1e12, "unit": "TFLOP/s (2 b m n per layer)",
+                                       "steps": k_var, "note": "forward GEMMs of the same layers with E4M3 operands (per-tensor scales), quantisation included; not part of the backward metric"}
+            del fwd
         # the fused-producer variant (dY transformed and rounded inside the GEMM kernels), a few steps: it is several times slower
         if g in (32, 64, 128) and all(l.b % 256 == 0 and l.m % 256 == 0 for l in layers):
             def step_fused():

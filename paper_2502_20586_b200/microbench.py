@@ -3,6 +3,7 @@
     python -m paper_2502_20586_b200.microbench gemm  M N K            [--iters 20] [--out fp32]
     python -m paper_2502_20586_b200.microbench quant ROWS COLS REDUCE_DIM G [--rounding 0] [--iters 20]
     python -m paper_2502_20586_b200.microbench backward B N M G       [--iters 20] [--bias] [--accumulate --out fp32]
+    python -m paper_2502_20586_b200.microbench forward B N M          [--iters 20]      (E4M3 forward pass)
 
 Operands are random codes/scales (gemm) or N(0,1) bf16 (quant, backward).  Between timed launches a buffer
 larger than L2 is rewritten so every launch starts with a cold L2.  Prints one JSON line.
@@ -39,7 +40,7 @@ def _time(fn, iters, flush_buf):
 
 def main(argv=None):
     ap = argparse.ArgumentParser()
-    ap.add_argument("kind", choices=["gemm", "quant", "backward"])
+    ap.add_argument("kind", choices=["gemm", "quant", "backward", "forward"])
     ap.add_argument("dims", type=int, nargs="+")
     ap.add_argument("--iters", type=int, default=20)
     ap.add_argument("--rounding", type=int, default=0)
@@ -75,6 +76,15 @@ def main(argv=None):
                           args.iters, flush)
         by = rows * cols * (2.0 + 0.5 + 1.0 / 32.0)
         res.update(ms=med, ms_best=best, gbs=by / med / 1e6, gbs_best=by / best / 1e6)
+    elif args.kind == "forward":
+        b, n, m = args.dims
+        x = torch.randn((b, n), generator=gen, device=dev).to(torch.bfloat16)
+        W = (torch.randn((m, n), generator=gen, device=dev) * 0.02).to(torch.bfloat16)
+        y = torch.empty((b, m), dtype=torch.float32 if out_dtype == mx.OUT_FP32 else torch.bfloat16, device=dev)
+        ws = torch.empty(int(mx.lib().mxfp4_linear_forward_fp8_workspace(b, n, m)), dtype=torch.uint8, device=dev)
+        med, best = _time(lambda: mx.mxfp4_linear_forward_fp8(x, W, out_dtype, y=y, workspace=ws), args.iters, flush)
+        fl = 2.0 * b * m * n
+        res.update(ms=med, ms_best=best, tflops=fl / med / 1e9, tflops_best=fl / best / 1e9)
     else:
         b, n, m, g = args.dims
         dY = torch.randn((b, m), generator=gen, device=dev).to(torch.bfloat16)
