@@ -487,6 +487,28 @@ def run_gpu(args):
             fl2 = sum(l.flops for l in lay2)
             other_configs[cfg] = {"value": fl2 / (ms2 * 1e-3) / 1e12, "unit": UNIT, "ms_per_step": ms2, "steps": 20, "g": g2,
                                   "frac_of_nominal_9pf": fl2 / (ms2 * 1e-3) / 1e12 / NOMINAL_FP4_TFLOPS}
+            # the same step captured once into a CUDA graph and replayed: these layers' kernels last 10-40 us, so the
+            # host's launch work (tensor-map encoding, three or four launches per call) shows in the eager number
+            try:
+                gs = torch.cuda.Stream(device=dev)
+                graph = torch.cuda.CUDAGraph()
+                with torch.cuda.stream(gs):
+                    with torch.cuda.graph(graph, stream=gs):
+                        step2()
+                for _ in range(5):
+                    graph.replay()
+                torch.cuda.synchronize()
+                a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+                a.record(stream)
+                for _ in range(20):
+                    graph.replay()
+                b.record(stream)
+                torch.cuda.synchronize()
+                msg = a.elapsed_time(b) / 20
+                other_configs[cfg]["cuda_graph"] = {"value": fl2 / (msg * 1e-3) / 1e12, "ms_per_step": msg, "steps": 20}
+                del graph
+            except RuntimeError as exc:                             # capture is a convenience of this leg, not part of the path
+                other_configs[cfg]["cuda_graph"] = {"error": str(exc)[:200]}
             del d2, ws2
     clocks = sampler.stop(n_timed)
     ms_e2e, h2d, d2h = None, 0, 0
