@@ -23,6 +23,8 @@
 // A-row scales are per CTA; every CTA needs the scales of all 256 B rows.
 #include <cuda_bf16.h>
 
+#include <cstdlib>
+
 #include "kernels.h"
 #include "ptx.cuh"
 
@@ -495,12 +497,15 @@ cudaError_t launch_gemm_pair(const GemmArgs& a, cudaStream_t stream) {
     // Tile order: groups of group_m pair-tile rows x all n-tiles.  Inside a group the A rows stay in L2 and B streams
     // through once; B is fetched from DRAM once for the whole launch only if it survives in L2 from one group to the
     // next, i.e. if a group's A rows + all of B + the group's output fit the part of L2 that behaves as one cache
-    // (about half of the 126 MB: 48 MB is used here).  Measured on 16384 x 4096 x 16384: 8 rows 348 MB of DRAM reads,
-    // 4 rows 243 MB, 2 rows 234 MB (operands: 168 MB), and +1 % speed.
+    // (about half of the 126 MB: 48 MB is used here).  Eight rows where that holds, else four: on 16384 x 4096 x 16384
+    // eight rows read 348 MB from DRAM, four 243 MB (operands: 168 MB) at the same speed inside a backward step;
+    // groups of two or one row read a little less still but cost 0.3 % / 2.5 % of the step (fewer pairs share a B tile
+    // at any moment).
     {
         const double b_bytes = (double)a.N * (double)a.K * 0.53125, out_b = a.out_fp32 ? 4.0 : 2.0;
-        int gm = 8;
-        while (gm > 1 && gm * 256.0 * (double)a.K * 0.53125 + b_bytes + gm * 256.0 * (double)a.N * out_b > 48.0 * 1024 * 1024) gm >>= 1;
+        int gm = 8.0 * 256.0 * (double)a.K * 0.53125 + b_bytes + 8.0 * 256.0 * (double)a.N * out_b > 48.0 * 1024 * 1024 ? 4 : 8;
+        const char* e = getenv("MXFP4_GEMM_GROUP_M");              // tuning switch: fixed group size (1..64) instead of the rule above
+        if (e != nullptr && atoi(e) >= 1 && atoi(e) <= 64) gm = atoi(e);
         p.group_m = gm;
     }
     cudaLaunchConfig_t cfg = {};
